@@ -1,0 +1,566 @@
+// C ABI of the ASD library: context life cycle, table construction, the host side of the round
+// driver (Algorithm 1's while loop), the sequential sampler (Eq. 7) and the diagnostics.
+#include <math.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <algorithm>
+#include <new>
+
+#include "asd_internal.h"
+
+using namespace asd;
+
+struct asd_ctx {
+  Ctx c;
+};
+
+namespace {
+
+thread_local std::string g_create_error;
+
+asd_status fail(Ctx* c, asd_status st, const std::string& msg) {
+  if (c) c->err = msg;
+  return st;
+}
+
+#define ASD_CUDA(c, expr)                                                                   \
+  do {                                                                                      \
+    cudaError_t e__ = (expr);                                                               \
+    if (e__ != cudaSuccess)                                                                 \
+      return fail((c), e__ == cudaErrorMemoryAllocation ? ASD_ERR_OOM : ASD_ERR_CUDA,       \
+                  std::string(#expr) + ": " + cudaGetErrorString(e__));                     \
+  } while (0)
+
+template <typename T>
+asd_status dev_alloc(Ctx* c, T** out, size_t count) {
+  void* p = nullptr;
+  const size_t bytes = std::max<size_t>(count, 1) * sizeof(T);
+  cudaError_t e = cudaMalloc(&p, bytes);
+  if (e != cudaSuccess) return fail(c, ASD_ERR_OOM, std::string("cudaMalloc: ") + cudaGetErrorString(e));
+  c->dev_allocs.push_back(p);
+  e = cudaMemsetAsync(p, 0, bytes, c->stream);
+  if (e != cudaSuccess) return fail(c, ASD_ERR_CUDA, std::string("cudaMemset: ") + cudaGetErrorString(e));
+  *out = static_cast<T*>(p);
+  return ASD_OK;
+}
+
+template <typename T>
+asd_status dev_upload(Ctx* c, const T** out, const std::vector<T>& host) {
+  T* p = nullptr;
+  asd_status st = dev_alloc(c, &p, host.size());
+  if (st != ASD_OK) return st;
+  if (!host.empty()) ASD_CUDA(c, cudaMemcpy(p, host.data(), host.size() * sizeof(T), cudaMemcpyHostToDevice));
+  *out = p;
+  return ASD_OK;
+}
+
+asd_status check_device_error(Ctx* c) {
+  // counters_host must have been refreshed and the stream synchronised by the caller
+  if (c->counters_host->err != 0) {
+    const int code = c->counters_host->err;
+    cudaMemsetAsync(&c->counters->err, 0, sizeof(int), c->stream);
+    return fail(c, (asd_status)code, "a bounded device-side wait ran out (kernel returned early)");
+  }
+  return ASD_OK;
+}
+
+asd_status sync_counters(Ctx* c) {
+  ASD_CUDA(c, cudaMemcpyAsync(c->counters_host, c->counters, sizeof(RoundCounters), cudaMemcpyDeviceToHost, c->stream));
+  ASD_CUDA(c, cudaStreamSynchronize(c->stream));
+  return check_device_error(c);
+}
+
+// One iteration of Algorithm 1's while loop for all active chains (window = 1, use_u = false is
+// one step of Eq. 7).  active_bound: host-side upper bound on the number of active chains.
+asd_status enqueue_round(Ctx* c, int window, bool use_u, int active_bound) {
+  if (active_bound <= 0) return ASD_OK;
+  launch_prep(c, window);
+  RowSet rs1{&c->counters->n_active, active_bound, c->y, c->act, c->step1, c->act};
+  RowSet rs2{&c->counters->rows2, active_bound * (window - 1), c->Yhat, nullptr, c->row_step, c->row_slot};
+  asd_status st = ASD_OK;
+  switch (c->kind) {
+    case ASD_DEN_GMM_ISO:
+      launch_gmm(c, rs1, c->v);
+      launch_draft(c, window);
+      launch_gmm(c, rs2, c->G);
+      break;
+    case ASD_DEN_GAUSS_LINEAR:
+      launch_gauss(c, rs1, c->v);
+      launch_draft(c, window);
+      launch_gauss(c, rs2, c->G);
+      break;
+    default:
+      launch_pack(c, rs1);
+      st = mlp_forward(c, rs1, c->v);
+      if (st != ASD_OK) return st;
+      launch_draft(c, window);
+      st = mlp_forward(c, rs2, c->G);
+      if (st != ASD_OK) return st;
+      break;
+  }
+  launch_verify(c, window, use_u);
+  ASD_CUDA(c, cudaGetLastError());
+  return ASD_OK;
+}
+
+struct HostTables {
+  std::vector<float> eta, sig, c1, c2, tt;
+};
+
+uint16_t bf16_bits_host(float f) {
+  uint32_t u;
+  memcpy(&u, &f, 4);
+  const uint32_t lsb = (u >> 16) & 1u;
+  u += 0x7FFFu + lsb;
+  return (uint16_t)(u >> 16);
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* asd_version(void) { return "asd-b200 0.1 (sm_100a)"; }
+
+const char* asd_last_error(const asd_ctx* ctx) {
+  if (!ctx) return g_create_error.c_str();
+  return ctx->c.err.c_str();
+}
+
+void asd_destroy(asd_ctx* ctx) {
+  if (!ctx) return;
+  Ctx* c = &ctx->c;
+  cudaStreamSynchronize(c->stream);
+  for (void* p : c->dev_allocs) cudaFree(p);
+  if (c->counters_host) cudaFreeHost(c->counters_host);
+  if (c->ev0) cudaEventDestroy(c->ev0);
+  if (c->ev1) cudaEventDestroy(c->ev1);
+  delete ctx;
+}
+
+asd_status asd_create(const asd_config* cfg, void* cuda_stream, asd_ctx** out) {
+  g_create_error.clear();
+  auto bad = [&](asd_status st, const char* msg) {
+    g_create_error = msg;
+    return st;
+  };
+  if (!cfg || !out) return bad(ASD_ERR_INVALID_ARG, "cfg and out must not be NULL");
+  *out = nullptr;
+  if (cfg->d < 1 || cfg->d > 65536) return bad(ASD_ERR_INVALID_ARG, "d must be in 1..65536");
+  if (cfg->K < 1) return bad(ASD_ERR_INVALID_ARG, "K must be >= 1");
+  if (cfg->window < 1 || cfg->window > kMaxWindow) return bad(ASD_ERR_INVALID_ARG, "window must be in 1..64");
+  if (cfg->max_chains < 1) return bad(ASD_ERR_INVALID_ARG, "max_chains must be >= 1");
+  if (!cfg->t) return bad(ASD_ERR_INVALID_ARG, "t must not be NULL");
+  if (!(cfg->t[0] >= 0.0)) return bad(ASD_ERR_INVALID_ARG, "t[0] must be >= 0");
+  for (int i = 0; i < cfg->K; ++i) {
+    if (!(cfg->t[i + 1] > cfg->t[i]) || !isfinite(cfg->t[i + 1]))
+      return bad(ASD_ERR_INVALID_ARG, "t must be finite and strictly increasing");
+    if (cfg->sigma2 && !(cfg->sigma2[i] > 0.0 && isfinite(cfg->sigma2[i])))
+      return bad(ASD_ERR_INVALID_ARG, "sigma2 must be finite and positive");
+  }
+  const long long max_rows_ll = (long long)cfg->max_chains * std::max(cfg->window - 1, 1);
+  if (max_rows_ll > (1ll << 30) || max_rows_ll * cfg->d > (1ll << 40))
+    return bad(ASD_ERR_INVALID_ARG, "max_chains * window * d too large");
+  const asd_denoiser& D = cfg->den;
+  switch (D.kind) {
+    case ASD_DEN_GMM_ISO:
+      if (D.n_comp < 1 || D.n_comp > 256 || !D.means || !D.weights || !(D.sigma > 0.f))
+        return bad(ASD_ERR_INVALID_ARG, "GMM: need 1..256 components, means, weights, sigma > 0");
+      for (int j = 0; j < D.n_comp; ++j)
+        if (!(D.weights[j] > 0.f)) return bad(ASD_ERR_INVALID_ARG, "GMM: weights must be positive");
+      break;
+    case ASD_DEN_GAUSS_LINEAR:
+      if (!D.mu0 || !D.Q || !D.lam) return bad(ASD_ERR_INVALID_ARG, "Gaussian: mu0, Q, lam required");
+      if (cfg->d > 4096) return bad(ASD_ERR_UNSUPPORTED, "Gaussian posterior mean supports d <= 4096");
+      for (int j = 0; j < cfg->d; ++j)
+        if (!(D.lam[j] >= 0.f)) return bad(ASD_ERR_INVALID_ARG, "Gaussian: eigenvalues must be >= 0");
+      break;
+    case ASD_DEN_RESMLP_BF16:
+      if (D.width < 8 || D.width % 8 || D.n_layers < 0 || D.d_cond < 0 || D.d_temb < 0 || D.d_temb % 2)
+        return bad(ASD_ERR_INVALID_ARG, "MLP: width must be a positive multiple of 8, d_temb even, sizes >= 0");
+      if (!D.W_in || !D.W_out || !D.b_in || !D.b_out || (D.n_layers > 0 && (!D.W_hid || !D.b_hid)))
+        return bad(ASD_ERR_INVALID_ARG, "MLP: weight and bias pointers required");
+      break;
+    default:
+      return bad(ASD_ERR_INVALID_ARG, "unknown denoiser kind");
+  }
+  int ndev = 0;
+  if (cudaGetDeviceCount(&ndev) != cudaSuccess || ndev < 1) return bad(ASD_ERR_CUDA, "no CUDA device");
+
+  asd_ctx* ctx = new (std::nothrow) asd_ctx();
+  if (!ctx) return bad(ASD_ERR_OOM, "host allocation failed");
+  Ctx* c = &ctx->c;
+  auto abandon = [&](asd_status st) {
+    g_create_error = c->err;
+    asd_destroy(ctx);
+    return st;
+  };
+  c->d = cfg->d;
+  c->K = cfg->K;
+  c->window = std::min(cfg->window, cfg->K);
+  c->max_chains = cfg->max_chains;
+  c->kind = D.kind;
+  c->seed = cfg->seed;
+  c->stream = static_cast<cudaStream_t>(cuda_stream);
+  c->max_rows = (int)((long long)cfg->max_chains * std::max(c->window - 1, 1));
+  cudaGetDevice(&c->device);
+  cudaDeviceProp prop;
+  if (cudaGetDeviceProperties(&prop, c->device) != cudaSuccess) return abandon(fail(c, ASD_ERR_CUDA, "device query failed"));
+  c->num_sms = prop.multiProcessorCount;
+  if (D.kind == ASD_DEN_RESMLP_BF16 && prop.major != 10)
+    return abandon(fail(c, ASD_ERR_UNSUPPORTED, "the bf16 network denoiser needs an sm_100 device (tcgen05 / TMEM)"));
+  if (cudaEventCreate(&c->ev0) != cudaSuccess || cudaEventCreate(&c->ev1) != cudaSuccess)
+    return abandon(fail(c, ASD_ERR_CUDA, "event creation failed"));
+  if (cudaMallocHost(&c->counters_host, sizeof(RoundCounters)) != cudaSuccess)
+    return abandon(fail(c, ASD_ERR_OOM, "pinned allocation failed"));
+  memset(c->counters_host, 0, sizeof(RoundCounters));
+
+  // ---- per-step tables: fp64 on the host, stored as fp32 -----------------------------------
+  const int K = c->K;
+  HostTables T;
+  T.eta.resize(K);
+  T.sig.resize(K);
+  T.c1.resize(K);
+  T.c2.resize(K);
+  T.tt.resize(K + 1);
+  for (int i = 0; i <= K; ++i) T.tt[i] = (float)cfg->t[i];
+  for (int i = 0; i < K; ++i) {
+    const double eta = cfg->t[i + 1] - cfg->t[i];
+    const double s2 = cfg->sigma2 ? cfg->sigma2[i] : eta;
+    const double sig = sqrt(s2);
+    T.eta[i] = (float)eta;
+    T.sig[i] = (float)sig;
+    T.c1[i] = (float)(eta / sig);
+    T.c2[i] = (float)(eta * eta / (2.0 * s2));
+  }
+  asd_status st;
+#define TRY(x)                          \
+  do {                                  \
+    st = (x);                           \
+    if (st != ASD_OK) return abandon(st); \
+  } while (0)
+  TRY(dev_upload(c, &c->tab.eta, T.eta));
+  TRY(dev_upload(c, &c->tab.sig, T.sig));
+  TRY(dev_upload(c, &c->tab.c1, T.c1));
+  TRY(dev_upload(c, &c->tab.c2, T.c2));
+  TRY(dev_upload(c, &c->tab.tt, T.tt));
+
+  // ---- state and workspaces --------------------------------------------------------------------
+  const size_t n = c->max_chains, d = c->d, R = c->max_rows;
+  TRY(dev_alloc(c, &c->y, n * d));
+  TRY(dev_alloc(c, &c->a, n));
+  TRY(dev_alloc(c, &c->rounds, n));
+  TRY(dev_alloc(c, &c->act, n));
+  TRY(dev_alloc(c, &c->row_off, n + 1));
+  TRY(dev_alloc(c, &c->step1, n));
+  TRY(dev_alloc(c, &c->row_step, R));
+  TRY(dev_alloc(c, &c->row_slot, R));
+  TRY(dev_alloc(c, &c->v, n * d));
+  TRY(dev_alloc(c, &c->Yhat, R * d));
+  TRY(dev_alloc(c, &c->G, R * d));
+  TRY(dev_alloc(c, &c->dbg_lr, n * c->window));
+  TRY(dev_alloc(c, &c->dbg_lu, n * c->window));
+  TRY(dev_alloc(c, &c->acc_len, n));
+  TRY(dev_alloc(c, &c->counters, 2));  // [0] round counters, [1].n_active doubles as a row-count scratch
+
+  // ---- denoiser parameters ---------------------------------------------------------------------
+  if (D.kind == ASD_DEN_GMM_ISO) {
+    std::vector<float> means(D.means, D.means + (size_t)D.n_comp * d), log_pi(D.n_comp), cnorm(D.n_comp);
+    double wsum = 0;
+    for (int j = 0; j < D.n_comp; ++j) wsum += D.weights[j];
+    for (int j = 0; j < D.n_comp; ++j) {
+      log_pi[j] = (float)log((double)D.weights[j] / wsum);
+      double s = 0;
+      for (size_t k = 0; k < d; ++k) s += (double)means[j * d + k] * means[j * d + k];
+      cnorm[j] = (float)s;
+    }
+    c->gmm.n_comp = D.n_comp;
+    c->gmm.s2 = (float)((double)D.sigma * (double)D.sigma);
+    TRY(dev_upload(c, &c->gmm.means, means));
+    TRY(dev_upload(c, &c->gmm.log_pi, log_pi));
+    TRY(dev_upload(c, &c->gmm.cnorm, cnorm));
+  } else if (D.kind == ASD_DEN_GAUSS_LINEAR) {
+    std::vector<float> Q(D.Q, D.Q + d * d), Qt(d * d), qmu(d), lam(D.lam, D.lam + d);
+    for (size_t i = 0; i < d; ++i)
+      for (size_t j = 0; j < d; ++j) Qt[j * d + i] = Q[i * d + j];
+    for (size_t j = 0; j < d; ++j) {
+      double s = 0;
+      for (size_t i = 0; i < d; ++i) s += (double)Q[i * d + j] * D.mu0[i];
+      qmu[j] = (float)s;
+    }
+    TRY(dev_upload(c, &c->gauss.Q, Q));
+    TRY(dev_upload(c, &c->gauss.Qt, Qt));
+    TRY(dev_upload(c, &c->gauss.qmu, qmu));
+    TRY(dev_upload(c, &c->gauss.lam, lam));
+  } else {
+    MlpParams& M = c->mlp;
+    M.d_cond = D.d_cond;
+    M.d_temb = D.d_temb;
+    M.width = D.width;
+    M.n_layers = D.n_layers;
+    M.in_dim = (int)d + D.d_cond + D.d_temb;
+    M.in_pad = (M.in_dim + 63) / 64 * 64;
+    M.row_cap = (int)std::max(R, n);
+    const size_t W = D.width;
+    std::vector<uint16_t> w_in((size_t)W * M.in_pad, 0);
+    for (size_t o = 0; o < W; ++o) memcpy(&w_in[o * M.in_pad], D.W_in + o * M.in_dim, (size_t)M.in_dim * 2);
+    std::vector<uint16_t> w_hid(D.W_hid ? D.W_hid : nullptr, D.W_hid ? D.W_hid + (size_t)D.n_layers * W * W : nullptr);
+    std::vector<uint16_t> w_out(D.W_out, D.W_out + d * W);
+    std::vector<float> b_in(D.b_in, D.b_in + W), b_out(D.b_out, D.b_out + d);
+    std::vector<float> b_hid(D.b_hid ? D.b_hid : nullptr, D.b_hid ? D.b_hid + (size_t)D.n_layers * W : nullptr);
+    std::vector<float> c_in(K, 1.f), c_skip(K, 0.f), c_out(K, 1.f);
+    if (D.c_in) c_in.assign(D.c_in, D.c_in + K);
+    if (D.c_skip) c_skip.assign(D.c_skip, D.c_skip + K);
+    if (D.c_out) c_out.assign(D.c_out, D.c_out + K);
+    std::vector<uint16_t> temb((size_t)K * D.d_temb);
+    const int half = D.d_temb / 2;
+    for (int i = 0; i < K; ++i) {
+      const double tau = 1000.0 * i / K;
+      for (int f = 0; f < half; ++f) {
+        const double w = exp(-log(1.0e4) * f / half);
+        temb[(size_t)i * D.d_temb + f] = bf16_bits_host((float)sin(tau * w));
+        temb[(size_t)i * D.d_temb + half + f] = bf16_bits_host((float)cos(tau * w));
+      }
+    }
+    TRY(dev_upload(c, reinterpret_cast<const uint16_t**>(&M.W_in), w_in));
+    TRY(dev_upload(c, reinterpret_cast<const uint16_t**>(&M.W_hid), w_hid));
+    TRY(dev_upload(c, reinterpret_cast<const uint16_t**>(&M.W_out), w_out));
+    TRY(dev_upload(c, &M.b_in, b_in));
+    TRY(dev_upload(c, &M.b_hid, b_hid));
+    TRY(dev_upload(c, &M.b_out, b_out));
+    TRY(dev_upload(c, &c->tab.c_in, c_in));
+    TRY(dev_upload(c, &c->tab.c_skip, c_skip));
+    TRY(dev_upload(c, &c->tab.c_out, c_out));
+    TRY(dev_upload(c, reinterpret_cast<const uint16_t**>(&M.temb), temb));
+    __nv_bfloat16* p = nullptr;
+    TRY(dev_alloc(c, &p, n * (size_t)D.d_cond));
+    M.cond = p;
+    TRY(dev_alloc(c, &c->cond_f32, n * (size_t)D.d_cond));
+    TRY(dev_alloc(c, &M.X, (size_t)M.row_cap * M.in_pad));
+    TRY(dev_alloc(c, &M.H[0], (size_t)M.row_cap * W));
+    TRY(dev_alloc(c, &M.H[1], (size_t)M.row_cap * W));
+  }
+#undef TRY
+  if (cudaStreamSynchronize(c->stream) != cudaSuccess) return abandon(fail(c, ASD_ERR_CUDA, "create: sync failed"));
+  *out = ctx;
+  return ASD_OK;
+}
+
+asd_status asd_reset(asd_ctx* ctx, int32_t n_chains, uint64_t chain_id_base, const float* y0_dev,
+                     const float* cond_dev) {
+  if (!ctx) return ASD_ERR_INVALID_ARG;
+  Ctx* c = &ctx->c;
+  if (n_chains < 0 || n_chains > c->max_chains) return fail(c, ASD_ERR_INVALID_ARG, "n_chains out of range");
+  if (chain_id_base + (uint64_t)n_chains > (1ull << 32)) return fail(c, ASD_ERR_INVALID_ARG, "chain ids must stay below 2^32");
+  const bool need_cond = c->kind == ASD_DEN_RESMLP_BF16 && c->mlp.d_cond > 0;
+  if (need_cond && !cond_dev && n_chains > 0) return fail(c, ASD_ERR_INVALID_ARG, "cond_dev required (d_cond > 0)");
+  c->n = n_chains;
+  c->chain_base = chain_id_base;
+  const size_t nd = (size_t)n_chains * c->d;
+  if (y0_dev)
+    ASD_CUDA(c, cudaMemcpyAsync(c->y, y0_dev, nd * sizeof(float), cudaMemcpyDeviceToDevice, c->stream));
+  else
+    ASD_CUDA(c, cudaMemsetAsync(c->y, 0, nd * sizeof(float), c->stream));
+  ASD_CUDA(c, cudaMemsetAsync(c->a, 0, (size_t)c->max_chains * sizeof(int), c->stream));
+  ASD_CUDA(c, cudaMemsetAsync(c->rounds, 0, (size_t)c->max_chains * sizeof(int), c->stream));
+  ASD_CUDA(c, cudaMemsetAsync(c->counters, 0, 2 * sizeof(RoundCounters), c->stream));
+  launch_fill_int(c, c->acc_len, c->max_chains, -1);
+  if (need_cond && n_chains > 0) {
+    ASD_CUDA(c, cudaMemcpyAsync(c->cond_f32, cond_dev, (size_t)n_chains * c->mlp.d_cond * sizeof(float),
+                                cudaMemcpyDeviceToDevice, c->stream));
+    launch_cond_to_bf16(c, n_chains);
+  }
+  ASD_CUDA(c, cudaGetLastError());
+  c->have_reset = true;
+  c->launches = 0;
+  return ASD_OK;
+}
+
+asd_status asd_round(asd_ctx* ctx, asd_round_stats* stats_host) {
+  if (!ctx) return ASD_ERR_INVALID_ARG;
+  Ctx* c = &ctx->c;
+  if (!c->have_reset) return fail(c, ASD_ERR_STATE, "asd_round before asd_reset");
+  asd_status st = enqueue_round(c, c->window, true, c->n);
+  if (st != ASD_OK) return st;
+  if (stats_host) {
+    st = sync_counters(c);
+    if (st != ASD_OK) return st;
+    const RoundCounters& h = *c->counters_host;
+    stats_host->n_active_before = h.n_active;
+    stats_host->n_active_after = h.n_active_after;
+    stats_host->rows_pass1 = h.n_active;
+    stats_host->rows_pass2 = h.rows2;
+    stats_host->accepted_total = (int64_t)h.accepted;
+  }
+  return ASD_OK;
+}
+
+static asd_status finish_run(Ctx* c, float* y_out_dev, int32_t* rounds_out_dev, asd_run_stats* stats, long long launches0,
+                             bool want_round_stats) {
+  if (y_out_dev)
+    ASD_CUDA(c, cudaMemcpyAsync(y_out_dev, c->y, (size_t)c->n * c->d * sizeof(float), cudaMemcpyDeviceToDevice, c->stream));
+  if (rounds_out_dev)
+    ASD_CUDA(c, cudaMemcpyAsync(rounds_out_dev, c->rounds, (size_t)c->n * sizeof(int), cudaMemcpyDeviceToDevice, c->stream));
+  ASD_CUDA(c, cudaEventRecord(c->ev1, c->stream));
+  asd_status st = sync_counters(c);
+  if (st != ASD_OK) return st;
+  if (stats) {
+    float ms = 0.f;
+    cudaEventElapsedTime(&ms, c->ev0, c->ev1);
+    stats->ms_total = ms;
+    stats->rows_total = (int64_t)c->counters_host->rows_total;
+    stats->launches = c->launches - launches0;
+    stats->rounds_max = 0;
+    stats->rounds_mean = 0.0;
+    if (want_round_stats && c->n > 0) {
+      std::vector<int> r(c->n);
+      ASD_CUDA(c, cudaMemcpy(r.data(), c->rounds, (size_t)c->n * sizeof(int), cudaMemcpyDeviceToHost));
+      long long sum = 0;
+      int mx = 0;
+      for (int v : r) {
+        sum += v;
+        mx = std::max(mx, v);
+      }
+      stats->rounds_max = mx;
+      stats->rounds_mean = (double)sum / c->n;
+    }
+  }
+  return ASD_OK;
+}
+
+asd_status asd_sample(asd_ctx* ctx, float* y_out_dev, int32_t* rounds_out_dev, asd_run_stats* stats_host) {
+  if (!ctx) return ASD_ERR_INVALID_ARG;
+  Ctx* c = &ctx->c;
+  if (!c->have_reset) return fail(c, ASD_ERR_STATE, "asd_sample before asd_reset");
+  const long long launches0 = c->launches;
+  ASD_CUDA(c, cudaEventRecord(c->ev0, c->stream));
+  int active = c->n;
+  // Every chain needs at least ceil(remaining / window) rounds and at most `remaining` (Theorem 3:
+  // the cursor strictly increases); the active count is read back once per round.
+  long long guard = (long long)c->K + 2;
+  while (active > 0 && guard-- > 0) {
+    asd_status st = enqueue_round(c, c->window, true, active);
+    if (st != ASD_OK) return st;
+    st = sync_counters(c);
+    if (st != ASD_OK) return st;
+    active = c->counters_host->n_active_after;
+  }
+  if (active > 0) return fail(c, ASD_ERR_STATE, "chains still active after K rounds");
+  return finish_run(c, y_out_dev, rounds_out_dev, stats_host, launches0, true);
+}
+
+asd_status asd_sequential_ddpm(asd_ctx* ctx, float* y_out_dev, asd_run_stats* stats_host) {
+  if (!ctx) return ASD_ERR_INVALID_ARG;
+  Ctx* c = &ctx->c;
+  if (!c->have_reset) return fail(c, ASD_ERR_STATE, "asd_sequential_ddpm before asd_reset");
+  const long long launches0 = c->launches;
+  int min_a = c->K;
+  if (c->n > 0) {
+    std::vector<int> a(c->n);
+    ASD_CUDA(c, cudaMemcpyAsync(a.data(), c->a, (size_t)c->n * sizeof(int), cudaMemcpyDeviceToHost, c->stream));
+    ASD_CUDA(c, cudaStreamSynchronize(c->stream));
+    for (int v : a) min_a = std::min(min_a, v);
+  }
+  ASD_CUDA(c, cudaEventRecord(c->ev0, c->stream));
+  for (int i = min_a; i < c->K; ++i) {
+    asd_status st = enqueue_round(c, 1, false, c->n);
+    if (st != ASD_OK) return st;
+  }
+  return finish_run(c, y_out_dev, nullptr, stats_host, launches0, true);
+}
+
+asd_status asd_sample_host(asd_ctx* ctx, int32_t n_chains, uint64_t chain_id_base, const float* y0_host,
+                           const float* cond_host, int32_t sequential, float* y_out_host, int32_t* rounds_out_host,
+                           asd_run_stats* stats_host) {
+  if (!ctx) return ASD_ERR_INVALID_ARG;
+  Ctx* c = &ctx->c;
+  if (n_chains < 0 || n_chains > c->max_chains) return fail(c, ASD_ERR_INVALID_ARG, "n_chains out of range");
+  if (!y_out_host && n_chains > 0) return fail(c, ASD_ERR_INVALID_ARG, "y_out_host must not be NULL");
+  const size_t nd = (size_t)n_chains * c->d;
+  // the library's own state / workspace rows serve as staging: y0 -> G (unused until the first
+  // round), cond -> cond_f32 (reset converts it in place)
+  const bool need_cond = c->kind == ASD_DEN_RESMLP_BF16 && c->mlp.d_cond > 0;
+  if (need_cond && !cond_host && n_chains > 0) return fail(c, ASD_ERR_INVALID_ARG, "cond_host required (d_cond > 0)");
+  if (y0_host) ASD_CUDA(c, cudaMemcpyAsync(c->G, y0_host, nd * sizeof(float), cudaMemcpyHostToDevice, c->stream));
+  float* cond_stage = nullptr;
+  if (need_cond && n_chains > 0) {
+    cond_stage = c->Yhat;  // max_rows * d >= n * d_cond is not guaranteed; check
+    if ((size_t)c->max_rows * c->d < (size_t)n_chains * c->mlp.d_cond)
+      return fail(c, ASD_ERR_UNSUPPORTED, "conditioning larger than the staging workspace");
+    ASD_CUDA(c, cudaMemcpyAsync(cond_stage, cond_host, (size_t)n_chains * c->mlp.d_cond * sizeof(float),
+                                cudaMemcpyHostToDevice, c->stream));
+  }
+  asd_status st = asd_reset(ctx, n_chains, chain_id_base, y0_host ? c->G : nullptr, cond_stage);
+  if (st != ASD_OK) return st;
+  st = sequential ? asd_sequential_ddpm(ctx, nullptr, stats_host) : asd_sample(ctx, nullptr, nullptr, stats_host);
+  if (st != ASD_OK) return st;
+  if (n_chains > 0) {
+    ASD_CUDA(c, cudaMemcpyAsync(y_out_host, c->y, nd * sizeof(float), cudaMemcpyDeviceToHost, c->stream));
+    if (rounds_out_host)
+      ASD_CUDA(c, cudaMemcpyAsync(rounds_out_host, c->rounds, (size_t)n_chains * sizeof(int), cudaMemcpyDeviceToHost, c->stream));
+    ASD_CUDA(c, cudaStreamSynchronize(c->stream));
+  }
+  return ASD_OK;
+}
+
+asd_status asd_get_state(asd_ctx* ctx, int32_t* a_dev, float* y_dev, int32_t* rounds_dev) {
+  if (!ctx) return ASD_ERR_INVALID_ARG;
+  Ctx* c = &ctx->c;
+  if (!c->have_reset) return fail(c, ASD_ERR_STATE, "asd_get_state before asd_reset");
+  if (a_dev) ASD_CUDA(c, cudaMemcpyAsync(a_dev, c->a, (size_t)c->n * sizeof(int), cudaMemcpyDeviceToDevice, c->stream));
+  if (y_dev) ASD_CUDA(c, cudaMemcpyAsync(y_dev, c->y, (size_t)c->n * c->d * sizeof(float), cudaMemcpyDeviceToDevice, c->stream));
+  if (rounds_dev)
+    ASD_CUDA(c, cudaMemcpyAsync(rounds_dev, c->rounds, (size_t)c->n * sizeof(int), cudaMemcpyDeviceToDevice, c->stream));
+  return ASD_OK;
+}
+
+asd_status asd_set_state(asd_ctx* ctx, const int32_t* a_dev, const float* y_dev, const int32_t* rounds_dev) {
+  if (!ctx) return ASD_ERR_INVALID_ARG;
+  Ctx* c = &ctx->c;
+  if (!c->have_reset) return fail(c, ASD_ERR_STATE, "asd_set_state before asd_reset");
+  if (a_dev) ASD_CUDA(c, cudaMemcpyAsync(c->a, a_dev, (size_t)c->n * sizeof(int), cudaMemcpyDeviceToDevice, c->stream));
+  if (y_dev) ASD_CUDA(c, cudaMemcpyAsync(c->y, y_dev, (size_t)c->n * c->d * sizeof(float), cudaMemcpyDeviceToDevice, c->stream));
+  if (rounds_dev)
+    ASD_CUDA(c, cudaMemcpyAsync(c->rounds, rounds_dev, (size_t)c->n * sizeof(int), cudaMemcpyDeviceToDevice, c->stream));
+  return ASD_OK;
+}
+
+asd_status asd_debug_last_round(asd_ctx* ctx, float* ln_ratio_dev, float* ln_u_dev, int32_t* accepted_dev) {
+  if (!ctx) return ASD_ERR_INVALID_ARG;
+  Ctx* c = &ctx->c;
+  if (!c->have_reset) return fail(c, ASD_ERR_STATE, "asd_debug_last_round before asd_reset");
+  const size_t nw = (size_t)c->n * c->window;
+  if (ln_ratio_dev) ASD_CUDA(c, cudaMemcpyAsync(ln_ratio_dev, c->dbg_lr, nw * sizeof(float), cudaMemcpyDeviceToDevice, c->stream));
+  if (ln_u_dev) ASD_CUDA(c, cudaMemcpyAsync(ln_u_dev, c->dbg_lu, nw * sizeof(float), cudaMemcpyDeviceToDevice, c->stream));
+  if (accepted_dev)
+    ASD_CUDA(c, cudaMemcpyAsync(accepted_dev, c->acc_len, (size_t)c->n * sizeof(int), cudaMemcpyDeviceToDevice, c->stream));
+  return ASD_OK;
+}
+
+asd_status asd_denoise(asd_ctx* ctx, int32_t n_rows, const int32_t* step_dev, const float* y_dev,
+                       const int32_t* slot_dev, float* out_dev) {
+  if (!ctx) return ASD_ERR_INVALID_ARG;
+  Ctx* c = &ctx->c;
+  if (n_rows < 0 || n_rows > c->max_rows) return fail(c, ASD_ERR_INVALID_ARG, "n_rows out of range");
+  if (n_rows == 0) return ASD_OK;
+  if (!step_dev || !y_dev || !out_dev) return fail(c, ASD_ERR_INVALID_ARG, "step_dev, y_dev, out_dev required");
+  const bool need_cond = c->kind == ASD_DEN_RESMLP_BF16 && c->mlp.d_cond > 0;
+  if (need_cond && !slot_dev) return fail(c, ASD_ERR_INVALID_ARG, "slot_dev required (d_cond > 0)");
+  int* n_dev = &c->counters[1].n_active;
+  ASD_CUDA(c, cudaMemcpyAsync(n_dev, &n_rows, sizeof(int), cudaMemcpyHostToDevice, c->stream));
+  RowSet rs{n_dev, n_rows, y_dev, nullptr, step_dev, slot_dev};
+  asd_status st = ASD_OK;
+  if (c->kind == ASD_DEN_GMM_ISO)
+    launch_gmm(c, rs, out_dev);
+  else if (c->kind == ASD_DEN_GAUSS_LINEAR)
+    launch_gauss(c, rs, out_dev);
+  else {
+    launch_pack(c, rs);
+    st = mlp_forward(c, rs, out_dev);
+    if (st != ASD_OK) return st;
+  }
+  ASD_CUDA(c, cudaGetLastError());
+  return sync_counters(c);
+}
+
+}  // extern "C"

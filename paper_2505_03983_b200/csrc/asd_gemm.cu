@@ -1,0 +1,491 @@
+// The network denoiser's forward pass as a chain of bf16 x bf16 -> fp32 GEMMs on the 5th-generation
+// tensor cores: operands staged in shared memory by TMA (128-byte swizzle), tcgen05.mma issued by one
+// thread with the accumulator in tensor memory, a warp-specialised persistent kernel (one TMA warp,
+// one MMA warp, four epilogue warps) with a multi-stage mbarrier pipeline and a double-buffered
+// accumulator so that the epilogue of one tile overlaps the MMAs of the next.
+//
+//   Y[m, n] = sum_k A[m, k] W[n, k]      A: activations [rows, K] row-major, W: weights [N, K] row-major
+//
+// Epilogues (fused, fp32 math on the un-rounded accumulator):
+//   EPI_IN   h_0 = bf16(acc + b)
+//   EPI_HID  h_l = bf16(h_{l-1} + SiLU(acc + b))
+//   EPI_OUT  g   = c_skip[i] y + c_out[i] (acc + b)          (fp32 store)
+//
+// Every wait on an mbarrier is bounded: when the limit runs out the thread records
+// ASD_ERR_TIMEOUT in the context's device error word and carries on as if the wait had
+// completed, so the kernel always reaches its tear-down (tensor memory is released) and the host
+// reports the error after the call.
+#include "asd_internal.h"
+
+namespace asd {
+
+namespace {
+
+constexpr int BM = 128;       // rows of an output tile = MMA M = tensor-memory lanes
+constexpr int BK = 64;        // bf16 elements per k-block = one 128-byte swizzle row
+constexpr int UMMA_K = 16;    // k extent of one tcgen05.mma (bf16)
+constexpr int kGemmThreads = 192;
+constexpr int kEpiWarp0 = 2;  // warps 2..5 are epilogue warps
+constexpr long long kWaitCycles = 400000000ll;  // ~0.2 s at 1.9 GHz per wait
+
+enum { EPI_IN = 0, EPI_HID = 1, EPI_OUT = 2 };
+
+struct GemmArgs {
+  int n_out;            // N
+  int k_dim;            // K (any; the TMA zero-fills beyond the tensor)
+  const int* m_dev;     // valid rows (device)
+  int m_cap;            // rows of the activation buffers
+  const float* bias;    // [N]
+  __nv_bfloat16* out_bf16;        // EPI_IN / EPI_HID: [m, ld_h]
+  const __nv_bfloat16* resid;     // EPI_HID: h_{l-1} [m, ld_h]
+  int ld_h;
+  float* out_f32;       // EPI_OUT: [m, d]
+  const float* ysrc;    // EPI_OUT: state rows [*, d]
+  const int* row_map;   // EPI_OUT: optional indirection into ysrc
+  const int* row_step;  // EPI_OUT: step index per row
+  const float* c_skip;
+  const float* c_out;
+  int* err;
+};
+
+// ---- PTX wrappers ---------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok;
+}
+// Bounded wait.  `dead` is a CTA-shared flag: once any wait has run out, later waits give up after
+// a few polls so the kernel drains quickly.
+__device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatile int* dead, int* err) {
+  if (mbar_try_wait(bar, parity)) return;
+  const long long t0 = clock64();
+  const long long limit = *dead ? 2000ll : kWaitCycles;
+  while (!mbar_try_wait(bar, parity)) {
+    if (clock64() - t0 > limit) {
+      *dead = 1;
+      atomicExch(err, (int)ASD_ERR_TIMEOUT);
+      return;
+    }
+  }
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];" ::"r"(dst),
+      "l"(map), "r"(bar), "r"(x), "r"(y)
+      : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                            uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %6, %7, %8}, p;\n\t}" ::"r"(d_tmem),
+      "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(0u), "r"(0u), "r"(0u), "r"(0u)
+      : "memory");
+}
+// 32 lanes x 32 consecutive fp32 columns: thread t of the warp receives lane (base + t).
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor of a K-major tile stored as rows of 128 bytes with the 128-byte
+// swizzle (what the TMA writes): start address, leading byte offset 1 (unused for swizzled K-major),
+// stride byte offset 1024 (8 rows x 128 B), descriptor version 1, layout type 2 (128-byte swizzle).
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((addr & 0x3FFFFu) >> 4);
+  d |= (uint64_t)1 << 16;
+  d |= (uint64_t)(1024 >> 4) << 32;
+  d |= (uint64_t)1 << 46;
+  d |= (uint64_t)2 << 61;
+  return d;
+}
+
+// Instruction descriptor, kind::f16: D fp32, A and B bf16, both K-major, M = 128, N = BN.
+template <int BN>
+__device__ __forceinline__ constexpr uint32_t instr_desc() {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+}
+
+template <int BN>
+struct Cfg {
+  static constexpr int kStageBytes = (BM + BN) * BK * 2;
+  static constexpr int kStages = (BN >= 256) ? 4 : (BN >= 128) ? 6 : (BN >= 64) ? 8 : 10;
+  static constexpr int kTmemCols = (2 * BN < 32) ? 32 : 2 * BN;  // two accumulators
+  static constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
+};
+
+__device__ __forceinline__ float silu(float z) { return z / (1.0f + __expf(-z)); }
+
+template <int BN, int EPI>
+__global__ void __launch_bounds__(kGemmThreads, 1)
+gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_w, const GemmArgs g) {
+  using C = Cfg<BN>;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t tiles = (raw + 1023u) & ~1023u;  // stage buffers, 1024-byte aligned for the swizzle
+  uint8_t* aux = smem_raw + (tiles - raw) + C::kStages * C::kStageBytes;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(aux);  // full[S], empty[S], acc_full[2], acc_empty[2]
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(aux + 8 * (2 * C::kStages + 4));
+  volatile int* dead = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  const uint32_t bar0 = smem_u32(bars);
+  auto full_bar = [&](int s) { return bar0 + 8u * s; };
+  auto empty_bar = [&](int s) { return bar0 + 8u * (C::kStages + s); };
+  auto accf_bar = [&](int b) { return bar0 + 8u * (2 * C::kStages + b); };
+  auto acce_bar = [&](int b) { return bar0 + 8u * (2 * C::kStages + 2 + b); };
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int m = min(*g.m_dev, g.m_cap);
+  const int tiles_m = (m + BM - 1) / BM;
+  const int tiles_n = (g.n_out + BN - 1) / BN;
+  const int n_tiles = tiles_m * tiles_n;
+  const int num_kb = (g.k_dim + BK - 1) / BK;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < C::kStages; ++s) {
+      mbar_init(full_bar(s), 1);
+      mbar_init(empty_bar(s), 1);
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(accf_bar(b), 1);
+      mbar_init(acce_bar(b), 4);
+    }
+    *dead = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                 "r"((uint32_t)C::kTmemCols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ---------------- TMA producer ----------------
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      for (int t = blockIdx.x; t < n_tiles; t += gridDim.x) {
+        const int m0 = (t / tiles_n) * BM, n0 = (t % tiles_n) * BN;
+        for (int kb = 0; kb < num_kb; ++kb) {
+          mbar_wait(empty_bar(stage), phase ^ 1u, dead, g.err);
+          const uint32_t sa = tiles + stage * C::kStageBytes;
+          const uint32_t sb = sa + BM * BK * 2;
+          mbar_expect_tx(full_bar(stage), (uint32_t)C::kStageBytes);
+          tma_load_2d(sa, &map_a, full_bar(stage), kb * BK, m0);
+          tma_load_2d(sb, &map_w, full_bar(stage), kb * BK, n0);
+          if (++stage == C::kStages) {
+            stage = 0;
+            phase ^= 1u;
+          }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------- MMA issuer ----------------
+    if (lane == 0) {
+      constexpr uint32_t idesc = instr_desc<BN>();
+      int stage = 0;
+      uint32_t phase = 0;
+      int it = 0;
+      for (int t = blockIdx.x; t < n_tiles; t += gridDim.x, ++it) {
+        const int acc = it & 1;
+        const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
+        mbar_wait(acce_bar(acc), acc_phase ^ 1u, dead, g.err);  // epilogue has drained this accumulator
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
+        for (int kb = 0; kb < num_kb; ++kb) {
+          mbar_wait(full_bar(stage), phase, dead, g.err);
+          tc_fence_after();
+          const uint32_t sa = tiles + stage * C::kStageBytes;
+          const uint32_t sb = sa + BM * BK * 2;
+          const uint64_t da = smem_desc_sw128(sa), db = smem_desc_sw128(sb);
+#pragma unroll
+          for (int k = 0; k < BK / UMMA_K; ++k) {
+            // advancing 16 bf16 = 32 bytes inside the swizzled row: +2 in the (address >> 4) field
+            tc_mma_bf16(d_tmem, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), idesc, (kb | k) != 0 ? 1u : 0u);
+          }
+          tc_commit(empty_bar(stage));  // frees the stage once these MMAs have read it
+          if (++stage == C::kStages) {
+            stage = 0;
+            phase ^= 1u;
+          }
+        }
+        tc_commit(accf_bar(acc));  // accumulator complete
+      }
+    }
+  } else {
+    // ---------------- epilogue warps ----------------
+    const int quarter = warp & 3;  // tensor-memory lanes [32 quarter, 32 quarter + 32)
+    int it = 0;
+    for (int t = blockIdx.x; t < n_tiles; t += gridDim.x, ++it) {
+      const int m0 = (t / tiles_n) * BM, n0 = (t % tiles_n) * BN;
+      const int acc = it & 1;
+      const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
+      mbar_wait(accf_bar(acc), acc_phase, dead, g.err);
+      tc_fence_after();
+      const int row = m0 + quarter * 32 + lane;
+      const bool row_ok = row < m;
+      float cs = 0.f, co = 0.f;
+      const float* ysrc_row = nullptr;
+      if (EPI == EPI_OUT && row_ok) {
+        const int step = g.row_step[row];
+        cs = g.c_skip[step];
+        co = g.c_out[step];
+        ysrc_row = g.ysrc + (size_t)(g.row_map ? g.row_map[row] : row) * g.n_out;
+      }
+#pragma unroll 1
+      for (int c0 = 0; c0 < BN; c0 += 32) {
+        uint32_t r[32];
+        const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN + c0);
+        tc_ld32(taddr, r);
+        tc_wait_ld();
+        const int col0 = n0 + c0;
+        if (row_ok && col0 < g.n_out) {
+          if (EPI == EPI_OUT) {
+            float* orow = g.out_f32 + (size_t)row * g.n_out;
+            const bool vec = (g.n_out % 4 == 0) && (col0 + 32 <= g.n_out);
+            if (vec) {
+#pragma unroll
+              for (int e = 0; e < 32; e += 4) {
+                const float4 b4 = *reinterpret_cast<const float4*>(g.bias + col0 + e);
+                const float4 y4 = *reinterpret_cast<const float4*>(ysrc_row + col0 + e);
+                float4 o;
+                o.x = fmaf(cs, y4.x, co * (__uint_as_float(r[e + 0]) + b4.x));
+                o.y = fmaf(cs, y4.y, co * (__uint_as_float(r[e + 1]) + b4.y));
+                o.z = fmaf(cs, y4.z, co * (__uint_as_float(r[e + 2]) + b4.z));
+                o.w = fmaf(cs, y4.w, co * (__uint_as_float(r[e + 3]) + b4.w));
+                *reinterpret_cast<float4*>(orow + col0 + e) = o;
+              }
+            } else {
+#pragma unroll
+              for (int e = 0; e < 32; ++e) {
+                const int col = col0 + e;
+                if (col < g.n_out)
+                  orow[col] = fmaf(cs, ysrc_row[col], co * (__uint_as_float(r[e]) + g.bias[col]));
+              }
+            }
+          } else {
+            __nv_bfloat16* orow = g.out_bf16 + (size_t)row * g.ld_h;
+            const __nv_bfloat16* rrow = (EPI == EPI_HID) ? g.resid + (size_t)row * g.ld_h : nullptr;
+            const bool vec = (g.ld_h % 8 == 0) && (col0 + 32 <= g.n_out);
+            if (vec) {
+#pragma unroll
+              for (int e = 0; e < 32; e += 8) {
+                float x[8];
+                const float4 b0 = *reinterpret_cast<const float4*>(g.bias + col0 + e);
+                const float4 b1 = *reinterpret_cast<const float4*>(g.bias + col0 + e + 4);
+                const float bb[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
+#pragma unroll
+                for (int u = 0; u < 8; ++u) x[u] = __uint_as_float(r[e + u]) + bb[u];
+                if (EPI == EPI_HID) {
+                  const uint4 rv = *reinterpret_cast<const uint4*>(rrow + col0 + e);
+                  const __nv_bfloat162* rp = reinterpret_cast<const __nv_bfloat162*>(&rv);
+#pragma unroll
+                  for (int u = 0; u < 4; ++u) {
+                    const float2 rf = __bfloat1622float2(rp[u]);
+                    x[2 * u] = rf.x + silu(x[2 * u]);
+                    x[2 * u + 1] = rf.y + silu(x[2 * u + 1]);
+                  }
+                }
+                uint4 ov;
+                __nv_bfloat162* op = reinterpret_cast<__nv_bfloat162*>(&ov);
+#pragma unroll
+                for (int u = 0; u < 4; ++u) op[u] = __floats2bfloat162_rn(x[2 * u], x[2 * u + 1]);
+                *reinterpret_cast<uint4*>(orow + col0 + e) = ov;
+              }
+            } else {
+#pragma unroll
+              for (int e = 0; e < 32; ++e) {
+                const int col = col0 + e;
+                if (col < g.n_out) {
+                  float x = __uint_as_float(r[e]) + g.bias[col];
+                  if (EPI == EPI_HID) x = __bfloat162float(rrow[col]) + silu(x);
+                  orow[col] = __float2bfloat16_rn(x);
+                }
+              }
+            }
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(acce_bar(acc));
+    }
+  }
+
+  // ---------------- tear-down ----------------
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)C::kTmemCols)
+                 : "memory");
+  }
+}
+
+// ---- host side --------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+
+// 2-D bf16 row-major tensor [rows, cols] (cols contiguous), box = [box_rows, 64 cols], 128-byte swizzle.
+bool get_tmap(Ctx* c, const void* ptr, int rows, int cols, int box_rows, CUtensorMap* out) {
+  auto key = std::make_tuple(ptr, rows, cols, box_rows);
+  auto it = c->tmaps.find(key);
+  if (it != c->tmaps.end()) {
+    *out = it->second;
+    return true;
+  }
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
+  cuuint32_t box[2] = {(cuuint32_t)BK, (cuuint32_t)box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  CUtensorMap m;
+  CUresult r = fn(&m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return false;
+  c->tmaps[key] = m;
+  *out = m;
+  return true;
+}
+
+template <int BN, int EPI>
+asd_status launch_gemm_t(Ctx* c, const void* a_ptr, int a_cols, const void* w_ptr, const GemmArgs& g, int m_bound) {
+  using C = Cfg<BN>;
+  CUtensorMap ma, mw;
+  if (!get_tmap(c, a_ptr, g.m_cap, a_cols, BM, &ma) || !get_tmap(c, w_ptr, g.n_out, a_cols, BN, &mw)) {
+    c->err = "cuTensorMapEncodeTiled failed";
+    return ASD_ERR_CUDA;
+  }
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaFuncSetAttribute(gemm_kernel<BN, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
+    attr_set = true;
+  }
+  const int tiles = ((m_bound + BM - 1) / BM) * ((g.n_out + BN - 1) / BN);
+  const int grid = tiles < c->num_sms ? (tiles < 1 ? 1 : tiles) : c->num_sms;
+  gemm_kernel<BN, EPI><<<grid, kGemmThreads, C::kSmemBytes, c->stream>>>(ma, mw, g);
+  c->launches++;
+  return ASD_OK;
+}
+
+template <int EPI>
+asd_status launch_gemm(Ctx* c, int bn, const void* a_ptr, int a_cols, const void* w_ptr, const GemmArgs& g,
+                       int m_bound) {
+  switch (bn) {
+    case 256: return launch_gemm_t<256, EPI>(c, a_ptr, a_cols, w_ptr, g, m_bound);
+    case 128: return launch_gemm_t<128, EPI>(c, a_ptr, a_cols, w_ptr, g, m_bound);
+    case 64: return launch_gemm_t<64, EPI>(c, a_ptr, a_cols, w_ptr, g, m_bound);
+    default: return launch_gemm_t<32, EPI>(c, a_ptr, a_cols, w_ptr, g, m_bound);
+  }
+}
+
+// Column-tile width: the widest tile that still gives every SM a tile.
+int pick_bn(const Ctx* c, int m_bound, int n_out) {
+  const int tiles_m = (m_bound + BM - 1) / BM;
+  const int cand[4] = {256, 128, 64, 32};
+  for (int i = 0; i < 4; ++i) {
+    const int bn = cand[i];
+    if (tiles_m * ((n_out + bn - 1) / bn) >= c->num_sms) return bn;
+  }
+  return 32;
+}
+
+}  // namespace
+
+asd_status mlp_forward(Ctx* c, const RowSet& rs, float* out) {
+  const MlpParams& M = c->mlp;
+  const int m_bound = rs.n_rows_max;
+  if (m_bound <= 0) return ASD_OK;
+  GemmArgs g{};
+  g.m_dev = rs.n_rows_dev;
+  g.m_cap = M.row_cap;
+  g.err = &c->counters->err;
+  asd_status st;
+  // input projection
+  g.n_out = M.width;
+  g.k_dim = M.in_pad;
+  g.bias = M.b_in;
+  g.out_bf16 = M.H[0];
+  g.ld_h = M.width;
+  const int bn_h = pick_bn(c, m_bound, M.width);
+  st = launch_gemm<EPI_IN>(c, bn_h, M.X, M.in_pad, M.W_in, g, m_bound);
+  if (st != ASD_OK) return st;
+  // residual layers
+  for (int l = 0; l < M.n_layers; ++l) {
+    g.k_dim = M.width;
+    g.bias = M.b_hid + (size_t)l * M.width;
+    g.resid = M.H[l & 1];
+    g.out_bf16 = M.H[(l + 1) & 1];
+    st = launch_gemm<EPI_HID>(c, bn_h, M.H[l & 1], M.width, M.W_hid + (size_t)l * M.width * M.width, g, m_bound);
+    if (st != ASD_OK) return st;
+  }
+  // output projection with the skip / scale epilogue
+  g.n_out = c->d;
+  g.k_dim = M.width;
+  g.bias = M.b_out;
+  g.out_bf16 = nullptr;
+  g.resid = nullptr;
+  g.out_f32 = out;
+  g.ysrc = rs.ysrc;
+  g.row_map = rs.row_map;
+  g.row_step = rs.row_step;
+  g.c_skip = c->tab.c_skip;
+  g.c_out = c->tab.c_out;
+  const int bn_o = pick_bn(c, m_bound, c->d);
+  return launch_gemm<EPI_OUT>(c, bn_o, M.H[M.n_layers & 1], M.width, M.W_out, g, m_bound);
+}
+
+}  // namespace asd

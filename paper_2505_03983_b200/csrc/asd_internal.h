@@ -1,0 +1,141 @@
+// Internal declarations shared by the translation units of the ASD library
+// (context layout, kernel launchers).  Nothing here crosses the C ABI.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <cuda.h>
+#include <stdint.h>
+
+#include <map>
+#include <string>
+#include <tuple>
+#include <vector>
+
+#include "asd.h"
+
+namespace asd {
+
+constexpr int kMaxWindow = 64;  // speculation length limit (two ballots in the verify kernel)
+
+// ---- device-side bookkeeping shared by all kernels of a round -------------------------
+// One small block of counters in device memory; the prep kernel rewrites it every round.
+struct RoundCounters {
+  int n_active;                 // chains with a < K at the start of the round
+  int rows2;                    // sum over active chains of (w - 1): rows of pass 2
+  int n_active_after;           // written by the verify kernel
+  int err;                      // device error word: 0, or ASD_ERR_TIMEOUT / ASD_ERR_STATE
+  unsigned long long accepted;  // steps advanced this round
+  unsigned long long rows_total;  // running total of drift evaluations since reset
+  unsigned long long pad[2];
+};
+
+// Per-step fp32 tables, built on the host in fp64 (asd_create).
+struct Tables {
+  const float* eta;    // [K]   eta_i = t_{i+1} - t_i
+  const float* sig;    // [K]   sigma_{i+1}
+  const float* c1;     // [K]   eta_i / sigma_{i+1}              (accept test, Algorithm 3)
+  const float* c2;     // [K]   eta_i^2 / (2 sigma_{i+1}^2)
+  const float* tt;     // [K+1] t_i
+  const float* c_in;   // [K]   (MLP) input scale
+  const float* c_skip; // [K]
+  const float* c_out;  // [K]
+};
+
+// Which rows a denoiser pass evaluates: point r is ysrc[row_map ? row_map[r] : r], at step
+// row_step[r], conditioned on chain position row_slot[r]; *n_rows_dev rows (<= n_rows_max).
+struct RowSet {
+  const int* n_rows_dev;
+  int n_rows_max;
+  const float* ysrc;
+  const int* row_map;
+  const int* row_step;
+  const int* row_slot;
+};
+
+struct GmmParams {
+  int n_comp;
+  const float* means;   // [n_comp, d]
+  const float* log_pi;  // [n_comp]
+  const float* cnorm;   // [n_comp] |c_j|^2
+  float s2;
+};
+
+struct GaussParams {
+  const float* Q;    // [d, d]   columns = eigenvectors
+  const float* Qt;   // [d, d]   transposed copy
+  const float* qmu;  // [d]      Q^T mu0
+  const float* lam;  // [d]
+};
+
+struct MlpParams {
+  int d_cond, d_temb, width, n_layers, in_dim, in_pad;
+  const __nv_bfloat16* W_in;   // [width, in_pad]  (zero padded columns)
+  const __nv_bfloat16* W_hid;  // [n_layers, width, width]
+  const __nv_bfloat16* W_out;  // [d, width]
+  const float* b_in;
+  const float* b_hid;
+  const float* b_out;
+  const __nv_bfloat16* temb;   // [K, d_temb]
+  const __nv_bfloat16* cond;   // [max_chains, d_cond]  bf16 copy made at reset
+  __nv_bfloat16* X;            // [row_cap, in_pad]
+  __nv_bfloat16* H[2];         // [row_cap, width]
+  int row_cap;
+};
+
+struct Ctx {
+  // configuration
+  int d = 0, K = 0, window = 0, max_chains = 0, kind = 0;
+  uint64_t seed = 0;
+  cudaStream_t stream = nullptr;
+  int device = 0;
+  int num_sms = 148;
+  // state
+  int n = 0;  // chains of the current reset
+  uint64_t chain_base = 0;
+  bool have_reset = false;
+  // device arrays
+  float* y = nullptr;        // [max_chains, d]
+  int* a = nullptr;          // [max_chains]
+  int* rounds = nullptr;     // [max_chains]
+  float* cond_f32 = nullptr; // [max_chains, d_cond]
+  int* act = nullptr;        // [max_chains] active position -> chain position
+  int* row_off = nullptr;    // [max_chains + 1]
+  int* step1 = nullptr;      // [max_chains] cursor of the active chain
+  int* row_step = nullptr;   // [max_rows] step of a pass-2 row
+  int* row_slot = nullptr;   // [max_rows] chain position of a pass-2 row
+  float* v = nullptr;        // [max_chains, d] drift at the current point, by active position
+  float* Yhat = nullptr;     // [max_rows, d] drafted points y^_{a+k}, k = 1..w-1
+  float* G = nullptr;        // [max_rows, d] drift at the drafted points
+  float* dbg_lr = nullptr;   // [max_chains, window]
+  float* dbg_lu = nullptr;   // [max_chains, window]
+  int* acc_len = nullptr;    // [max_chains]
+  RoundCounters* counters = nullptr;
+  RoundCounters* counters_host = nullptr;  // pinned
+  int max_rows = 0;
+  Tables tab{};
+  GmmParams gmm{};
+  GaussParams gauss{};
+  MlpParams mlp{};
+  std::vector<void*> dev_allocs;
+  std::map<std::tuple<const void*, int, int, int>, CUtensorMap> tmaps;
+  std::string err;
+  long long launches = 0;
+  cudaEvent_t ev0 = nullptr, ev1 = nullptr;
+};
+
+// ---- launchers (asd_kernels.cu) ---------------------------------------------------------
+void launch_prep(Ctx* c, int window);
+void launch_draft(Ctx* c, int window);
+void launch_verify(Ctx* c, int window, bool use_u);
+void launch_pack(Ctx* c, const RowSet& rs);
+void launch_gmm(Ctx* c, const RowSet& rs, float* out);
+void launch_gauss(Ctx* c, const RowSet& rs, float* out);
+void launch_cond_to_bf16(Ctx* c, int n);
+void launch_fill_int(Ctx* c, int* p, int n, int val);
+
+// ---- MLP forward (asd_gemm.cu) ----------------------------------------------------------
+// Runs the GEMM chain on the rows already packed into mlp.X; writes out[r] for r < *n_rows_dev.
+asd_status mlp_forward(Ctx* c, const RowSet& rs, float* out);
+
+}  // namespace asd

@@ -1,0 +1,609 @@
+// Elementwise / reduction kernels of the ASD round: bookkeeping (active list, row offsets),
+// draft (Algorithm 1, proposal loop), verify + resample + advance (Algorithms 2 and 3, and the
+// advance step of Algorithm 1), the closed-form posterior means (Eq. 4) and the feature packing
+// of the network denoiser.  fp32 throughout; no fast-math.
+#include "asd_internal.h"
+
+namespace asd {
+
+// ---------------------------------------------------------------------------------------------
+// Counter-based randomness (Algorithm 1, "sample u, xi"): Philox4x32-10, counter =
+// (dimension block, step, chain id, tag).
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint4 philox4x32_10(uint4 c, uint32_t k0, uint32_t k1) {
+  constexpr uint32_t M0 = 0xD2511F53u, M1 = 0xCD9E8D57u, W0 = 0x9E3779B9u, W1 = 0xBB67AE85u;
+#pragma unroll
+  for (int r = 0; r < 10; ++r) {
+    const uint32_t hi0 = __umulhi(M0, c.x), lo0 = M0 * c.x;
+    const uint32_t hi1 = __umulhi(M1, c.z), lo1 = M1 * c.z;
+    c = make_uint4(hi1 ^ c.y ^ k0, lo1, hi0 ^ c.w ^ k1, lo0);
+    k0 += W0;
+    k1 += W1;
+  }
+  return c;
+}
+
+__device__ __forceinline__ float uniform_from_word(uint32_t r) {
+  return (__uint2float_rn(r >> 9) + 0.5f) * 1.1920928955078125e-07f;  // 2^-23, exact
+}
+
+__device__ __forceinline__ void box_muller(uint32_t r_even, uint32_t r_odd, float& n_even, float& n_odd) {
+  const float rad = sqrtf(-2.0f * logf(uniform_from_word(r_even)));
+  float s, c;
+  sincospif(2.0f * uniform_from_word(r_odd), &s, &c);
+  n_even = rad * c;
+  n_odd = rad * s;
+}
+
+// xi_step[4q .. 4q+3]
+__device__ __forceinline__ float4 xi4(uint32_t q, uint32_t step, uint32_t chain, uint32_t k0, uint32_t k1) {
+  const uint4 r = philox4x32_10(make_uint4(q, step, chain, 0u), k0, k1);
+  float4 n;
+  box_muller(r.x, r.y, n.x, n.y);
+  box_muller(r.z, r.w, n.z, n.w);
+  return n;
+}
+
+__device__ __forceinline__ float ln_u(uint32_t step, uint32_t chain, uint32_t k0, uint32_t k1) {
+  const uint4 r = philox4x32_10(make_uint4(0u, step, chain, 1u), k0, k1);
+  return logf(uniform_from_word(r.x));
+}
+
+// Loads / stores of the 4 dims of block q with a ragged tail (d not a multiple of 4).
+__device__ __forceinline__ float4 load4(const float* row, int q, int d, bool vec) {
+  if (vec) return *reinterpret_cast<const float4*>(row + 4 * q);
+  float4 r = make_float4(0.f, 0.f, 0.f, 0.f);
+  const int b = 4 * q;
+  if (b + 0 < d) r.x = row[b + 0];
+  if (b + 1 < d) r.y = row[b + 1];
+  if (b + 2 < d) r.z = row[b + 2];
+  if (b + 3 < d) r.w = row[b + 3];
+  return r;
+}
+
+__device__ __forceinline__ void store4(float* row, int q, int d, bool vec, float4 val) {
+  if (vec) {
+    *reinterpret_cast<float4*>(row + 4 * q) = val;
+    return;
+  }
+  const int b = 4 * q;
+  if (b + 0 < d) row[b + 0] = val.x;
+  if (b + 1 < d) row[b + 1] = val.y;
+  if (b + 2 < d) row[b + 2] = val.z;
+  if (b + 3 < d) row[b + 3] = val.w;
+}
+
+__device__ __forceinline__ float warp_sum(float x) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
+  return x;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Round driver bookkeeping: compact the chains with a < K into the active list and lay out the
+// pass-2 rows (exclusive scan of w - 1).  One block; n is at most a few tens of thousands.
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(1024) prep_kernel(const int* __restrict__ a, int n, int K, int window,
+                                                    int* __restrict__ act, int* __restrict__ row_off,
+                                                    int* __restrict__ step1, int* __restrict__ acc_len,
+                                                    RoundCounters* __restrict__ cnt) {
+  __shared__ int s_cnt[32], s_rows[32];
+  __shared__ int s_base_cnt, s_base_rows;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  if (tid == 0) {
+    s_base_cnt = 0;
+    s_base_rows = 0;
+  }
+  __syncthreads();
+  for (int j0 = 0; j0 < n; j0 += blockDim.x) {
+    const int j = j0 + tid;
+    int aj = K, flag = 0, rows = 0;
+    if (j < n) {
+      aj = a[j];
+      flag = aj < K;
+      rows = flag ? min(window, K - aj) - 1 : 0;
+      acc_len[j] = -1;
+    }
+    // inclusive warp scans
+    int c = flag, r = rows;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int c2 = __shfl_up_sync(0xffffffffu, c, o);
+      const int r2 = __shfl_up_sync(0xffffffffu, r, o);
+      if (lane >= o) {
+        c += c2;
+        r += r2;
+      }
+    }
+    if (lane == 31) {
+      s_cnt[warp] = c;
+      s_rows[warp] = r;
+    }
+    __syncthreads();
+    if (warp == 0) {
+      int wc = s_cnt[lane], wr = s_rows[lane];
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int c2 = __shfl_up_sync(0xffffffffu, wc, o);
+        const int r2 = __shfl_up_sync(0xffffffffu, wr, o);
+        if (lane >= o) {
+          wc += c2;
+          wr += r2;
+        }
+      }
+      s_cnt[lane] = wc;
+      s_rows[lane] = wr;
+    }
+    __syncthreads();
+    const int pos = s_base_cnt + (warp ? s_cnt[warp - 1] : 0) + c - flag;
+    const int roff = s_base_rows + (warp ? s_rows[warp - 1] : 0) + r - rows;
+    if (flag) {
+      act[pos] = j;
+      row_off[pos] = roff;
+      step1[pos] = aj;
+    }
+    __syncthreads();
+    if (tid == 0) {
+      s_base_cnt += s_cnt[31];
+      s_base_rows += s_rows[31];
+    }
+    __syncthreads();
+  }
+  if (tid == 0) {
+    row_off[s_base_cnt] = s_base_rows;
+    cnt->n_active = s_base_cnt;
+    cnt->rows2 = s_base_rows;
+    cnt->n_active_after = 0;
+    cnt->accepted = 0ull;
+    cnt->rows_total += (unsigned long long)(s_base_cnt + s_base_rows);
+  }
+}
+
+void launch_prep(Ctx* c, int window) {
+  prep_kernel<<<1, 1024, 0, c->stream>>>(c->a, c->n, c->K, window, c->act, c->row_off, c->step1, c->acc_len,
+                                         c->counters);
+  c->launches++;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Draft (Algorithm 1, proposal loop): y^_{a+k} = y^_{a+k-1} + eta v_a + sigma xi_{a+k} for
+// k = 1..w-1 (the last proposal sample is only needed when the whole window is accepted and is
+// rebuilt by the verify kernel).  One thread owns 4 dims of one chain and walks the window, so the
+// "prefix sum" of the paper is a register recurrence.  Writes the fp32 points and, for the
+// network denoiser, its bf16 input rows.
+// ---------------------------------------------------------------------------------------------
+struct DraftArgs {
+  int d, K, window, nq, vec;
+  uint32_t k0, k1;
+  uint64_t chain_base;
+  const RoundCounters* cnt;
+  const int* act;
+  const int* a;
+  const int* row_off;
+  const float* y;
+  const float* v;
+  Tables tab;
+  float* Yhat;
+  int* row_step;
+  int* row_slot;
+  // network input rows (null for the closed-form denoisers)
+  __nv_bfloat16* X;
+  int in_pad, in_dim, d_cond, d_temb;
+  const __nv_bfloat16* cond;
+  const __nv_bfloat16* temb;
+};
+
+__global__ void __launch_bounds__(256) draft_kernel(const DraftArgs A) {
+  const int p = blockIdx.y;
+  if (p >= A.cnt->n_active) return;
+  const int j = A.act[p];
+  const int a = A.a[j];
+  const int w = min(A.window, A.K - a);
+  const int row0 = A.row_off[p];
+  const uint32_t chain = (uint32_t)(A.chain_base + (uint64_t)j);
+  const int q = blockIdx.x * blockDim.x + threadIdx.x;
+  if (q < A.nq) {
+    float4 yh = load4(A.y + (size_t)j * A.d, q, A.d, A.vec);
+    const float4 v = load4(A.v + (size_t)p * A.d, q, A.d, A.vec);
+    for (int k = 1; k < w; ++k) {
+      const int i = a + k - 1;  // step i -> i+1 uses eta_i, sigma_{i+1}, xi_{i+1}
+      const float eta = A.tab.eta[i], sig = A.tab.sig[i];
+      const float4 xi = xi4((uint32_t)q, (uint32_t)(i + 1), chain, A.k0, A.k1);
+      yh.x = fmaf(sig, xi.x, fmaf(eta, v.x, yh.x));
+      yh.y = fmaf(sig, xi.y, fmaf(eta, v.y, yh.y));
+      yh.z = fmaf(sig, xi.z, fmaf(eta, v.z, yh.z));
+      yh.w = fmaf(sig, xi.w, fmaf(eta, v.w, yh.w));
+      const int row = row0 + k - 1;
+      store4(A.Yhat + (size_t)row * A.d, q, A.d, A.vec, yh);
+      if (A.X) {
+        const float ci = A.tab.c_in[a + k];
+        __nv_bfloat16* xr = A.X + (size_t)row * A.in_pad + 4 * q;
+        if (A.vec) {
+          __nv_bfloat162 lo = __floats2bfloat162_rn(ci * yh.x, ci * yh.y);
+          __nv_bfloat162 hi = __floats2bfloat162_rn(ci * yh.z, ci * yh.w);
+          uint2 pk;
+          pk.x = *reinterpret_cast<uint32_t*>(&lo);
+          pk.y = *reinterpret_cast<uint32_t*>(&hi);
+          *reinterpret_cast<uint2*>(xr) = pk;
+        } else {
+          const int b = 4 * q;
+          if (b + 0 < A.d) xr[0] = __float2bfloat16_rn(ci * yh.x);
+          if (b + 1 < A.d) xr[1] = __float2bfloat16_rn(ci * yh.y);
+          if (b + 2 < A.d) xr[2] = __float2bfloat16_rn(ci * yh.z);
+          if (b + 3 < A.d) xr[3] = __float2bfloat16_rn(ci * yh.w);
+        }
+      }
+      if (q == 0) {
+        A.row_step[row] = a + k;
+        A.row_slot[row] = j;
+      }
+    }
+  }
+  // conditioning, time embedding and zero padding of the network input rows
+  if (A.X && blockIdx.x == 0) {
+    const int extra = A.in_pad - A.d;
+    for (int k = 1; k < w; ++k) {
+      const int row = row0 + k - 1;
+      __nv_bfloat16* xr = A.X + (size_t)row * A.in_pad + A.d;
+      for (int e = threadIdx.x; e < extra; e += blockDim.x) {
+        __nv_bfloat16 val = __float2bfloat16_rn(0.f);
+        if (e < A.d_cond)
+          val = A.cond[(size_t)j * A.d_cond + e];
+        else if (e < A.d_cond + A.d_temb)
+          val = A.temb[(size_t)(a + k) * A.d_temb + (e - A.d_cond)];
+        xr[e] = val;
+      }
+    }
+  }
+}
+
+void launch_draft(Ctx* c, int window) {
+  if (window <= 1 || c->n == 0) return;
+  DraftArgs A{};
+  A.d = c->d;
+  A.K = c->K;
+  A.window = window;
+  A.nq = (c->d + 3) / 4;
+  A.vec = (c->d % 4 == 0);
+  A.k0 = (uint32_t)(c->seed & 0xffffffffull);
+  A.k1 = (uint32_t)(c->seed >> 32);
+  A.chain_base = c->chain_base;
+  A.cnt = c->counters;
+  A.act = c->act;
+  A.a = c->a;
+  A.row_off = c->row_off;
+  A.y = c->y;
+  A.v = c->v;
+  A.tab = c->tab;
+  A.Yhat = c->Yhat;
+  A.row_step = c->row_step;
+  A.row_slot = c->row_slot;
+  if (c->kind == ASD_DEN_RESMLP_BF16) {
+    A.X = c->mlp.X;
+    A.in_pad = c->mlp.in_pad;
+    A.in_dim = c->mlp.in_dim;
+    A.d_cond = c->mlp.d_cond;
+    A.d_temb = c->mlp.d_temb;
+    A.cond = c->mlp.cond;
+    A.temb = c->mlp.temb;
+  }
+  const int threads = A.nq >= 256 ? 256 : (A.nq >= 128 ? 128 : 64);
+  dim3 grid((A.nq + threads - 1) / threads, c->n);
+  draft_kernel<<<grid, threads, 0, c->stream>>>(A);
+  c->launches++;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Verify + resample + advance (Algorithm 2, Algorithm 3, advance step of Algorithm 1).
+// One block per active chain.  Phase 1: one warp per window slot k >= 2 regenerates xi_{a+k},
+// reads the drift g_{k-1} at the drafted point once (coalesced float4) and reduces
+//   <xi, delta>, |delta|^2, delta = v_a - g_{k-1}      (m^ - m = eta delta)
+// over d with warp shuffles; ln ratio = -(eta/sigma) <xi, delta> - (eta^2 / 2 sigma^2) |delta|^2.
+// Phase 2: a ballot over the accept bits gives the all-accepted prefix length n.
+// Phase 3: the block writes the new state: the reflected sample at the first rejected slot
+//   y = y^_n + eta g_n + sigma (xi - 2 delta <delta, xi> / |delta|^2)
+// or, if everything was accepted, the last proposal sample y^_w.
+// ---------------------------------------------------------------------------------------------
+struct VerifyArgs {
+  int d, K, window, nq, vec, use_u;
+  uint32_t k0, k1;
+  uint64_t chain_base;
+  RoundCounters* cnt;
+  const int* act;
+  int* a;
+  int* rounds;
+  const int* row_off;
+  float* y;
+  const float* v;
+  const float* Yhat;
+  const float* G;
+  Tables tab;
+  float* dbg_lr;
+  float* dbg_lu;
+  int* acc_len;
+};
+
+__global__ void __launch_bounds__(256) verify_kernel(const VerifyArgs A) {
+  __shared__ float s_dot[kMaxWindow + 1], s_nrm[kMaxWindow + 1];
+  __shared__ int s_acc[kMaxWindow + 1];
+  __shared__ int s_n;
+  const int p = blockIdx.x;
+  if (p >= A.cnt->n_active) return;
+  const int j = A.act[p];
+  const int a = A.a[j];
+  const int w = min(A.window, A.K - a);
+  const int row0 = A.row_off[p];
+  const uint32_t chain = (uint32_t)(A.chain_base + (uint64_t)j);
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
+  const float* vrow = A.v + (size_t)p * A.d;
+
+  if (tid == 0) {
+    // slot 1: proposal mean == target mean, ratio exactly 1 (Lemma 1)
+    s_acc[1] = 1;
+    A.dbg_lr[(size_t)j * A.window] = 0.f;
+    A.dbg_lu[(size_t)j * A.window] = A.use_u ? ln_u((uint32_t)(a + 1), chain, A.k0, A.k1) : 0.f;
+  }
+  for (int k = 2 + warp; k <= w; k += nwarps) {
+    const float* grow = A.G + (size_t)(row0 + k - 2) * A.d;
+    float dot = 0.f, nrm = 0.f;
+    for (int q = lane; q < A.nq; q += 32) {
+      const float4 v = load4(vrow, q, A.d, A.vec);
+      const float4 g = load4(grow, q, A.d, A.vec);
+      const float4 xi = xi4((uint32_t)q, (uint32_t)(a + k), chain, A.k0, A.k1);
+      float4 dl = make_float4(v.x - g.x, v.y - g.y, v.z - g.z, v.w - g.w);
+      if (!A.vec) {  // ragged tail: dims >= d contribute nothing
+        const int b = 4 * q;
+        if (b + 1 >= A.d) dl.y = 0.f;
+        if (b + 2 >= A.d) dl.z = 0.f;
+        if (b + 3 >= A.d) dl.w = 0.f;
+      }
+      dot = fmaf(xi.x, dl.x, dot);
+      dot = fmaf(xi.y, dl.y, dot);
+      dot = fmaf(xi.z, dl.z, dot);
+      dot = fmaf(xi.w, dl.w, dot);
+      nrm = fmaf(dl.x, dl.x, nrm);
+      nrm = fmaf(dl.y, dl.y, nrm);
+      nrm = fmaf(dl.z, dl.z, nrm);
+      nrm = fmaf(dl.w, dl.w, nrm);
+    }
+    dot = warp_sum(dot);
+    nrm = warp_sum(nrm);
+    if (lane == 0) {
+      const int i = a + k - 1;
+      const float lr = -A.tab.c1[i] * dot - A.tab.c2[i] * nrm;
+      const float lu = ln_u((uint32_t)(a + k), chain, A.k0, A.k1);
+      s_dot[k] = dot;
+      s_nrm[k] = nrm;
+      s_acc[k] = (lu <= fminf(0.f, lr)) || (nrm == 0.f);
+      A.dbg_lr[(size_t)j * A.window + k - 1] = lr;
+      A.dbg_lu[(size_t)j * A.window + k - 1] = lu;
+    }
+  }
+  __syncthreads();
+  if (warp == 0) {
+    // first rejected slot: ballot over slots 1..32 and 33..64
+    const int k_lo = lane + 1, k_hi = lane + 33;
+    const unsigned rej_lo = __ballot_sync(0xffffffffu, k_lo <= w && !s_acc[k_lo]);
+    const unsigned rej_hi = __ballot_sync(0xffffffffu, k_hi <= w && !s_acc[k_hi]);
+    int n = w;
+    if (rej_lo)
+      n = __ffs(rej_lo) - 1;  // slot index of first reject is ffs, prefix length is one less
+    else if (rej_hi)
+      n = 32 + __ffs(rej_hi) - 1;
+    if (lane == 0) s_n = n;
+  }
+  __syncthreads();
+  const int n = s_n;
+  float* yrow = A.y + (size_t)j * A.d;
+  if (n < w) {
+    // reject at slot n + 1: target mean m = y^_n + eta g_n, reflected noise
+    const int i = a + n;
+    const float eta = A.tab.eta[i], sig = A.tab.sig[i];
+    const float coef = 2.f * s_dot[n + 1] / s_nrm[n + 1];
+    const float* base = A.Yhat + (size_t)(row0 + n - 1) * A.d;  // n >= 1 always
+    const float* grow = A.G + (size_t)(row0 + n - 1) * A.d;
+    for (int q = tid; q < A.nq; q += blockDim.x) {
+      const float4 b = load4(base, q, A.d, A.vec);
+      const float4 g = load4(grow, q, A.d, A.vec);
+      const float4 v = load4(vrow, q, A.d, A.vec);
+      const float4 xi = xi4((uint32_t)q, (uint32_t)(i + 1), chain, A.k0, A.k1);
+      float4 o;
+      o.x = fmaf(sig, fmaf(-coef, v.x - g.x, xi.x), fmaf(eta, g.x, b.x));
+      o.y = fmaf(sig, fmaf(-coef, v.y - g.y, xi.y), fmaf(eta, g.y, b.y));
+      o.z = fmaf(sig, fmaf(-coef, v.z - g.z, xi.z), fmaf(eta, g.z, b.z));
+      o.w = fmaf(sig, fmaf(-coef, v.w - g.w, xi.w), fmaf(eta, g.w, b.w));
+      store4(yrow, q, A.d, A.vec, o);
+    }
+  } else {
+    // whole window accepted: y_{a+w} = y^_{w-1} + eta v_a + sigma xi_{a+w}
+    const int i = a + w - 1;
+    const float eta = A.tab.eta[i], sig = A.tab.sig[i];
+    const float* base = (w == 1) ? yrow : A.Yhat + (size_t)(row0 + w - 2) * A.d;
+    for (int q = tid; q < A.nq; q += blockDim.x) {
+      const float4 b = load4(base, q, A.d, A.vec);
+      const float4 v = load4(vrow, q, A.d, A.vec);
+      const float4 xi = xi4((uint32_t)q, (uint32_t)(i + 1), chain, A.k0, A.k1);
+      float4 o;
+      o.x = fmaf(sig, xi.x, fmaf(eta, v.x, b.x));
+      o.y = fmaf(sig, xi.y, fmaf(eta, v.y, b.y));
+      o.z = fmaf(sig, xi.z, fmaf(eta, v.z, b.z));
+      o.w = fmaf(sig, xi.w, fmaf(eta, v.w, b.w));
+      store4(yrow, q, A.d, A.vec, o);
+    }
+  }
+  if (tid == 0) {
+    const int adv = (n < w) ? n + 1 : w;
+    A.a[j] = a + adv;
+    A.rounds[j] += 1;
+    A.acc_len[j] = n;
+    atomicAdd(&A.cnt->accepted, (unsigned long long)adv);
+    if (a + adv < A.K) atomicAdd(&A.cnt->n_active_after, 1);
+  }
+}
+
+void launch_verify(Ctx* c, int window, bool use_u) {
+  if (c->n == 0) return;
+  VerifyArgs A{};
+  A.d = c->d;
+  A.K = c->K;
+  A.window = window;
+  A.nq = (c->d + 3) / 4;
+  A.vec = (c->d % 4 == 0);
+  A.use_u = use_u;
+  A.k0 = (uint32_t)(c->seed & 0xffffffffull);
+  A.k1 = (uint32_t)(c->seed >> 32);
+  A.chain_base = c->chain_base;
+  A.cnt = c->counters;
+  A.act = c->act;
+  A.a = c->a;
+  A.rounds = c->rounds;
+  A.row_off = c->row_off;
+  A.y = c->y;
+  A.v = c->v;
+  A.Yhat = c->Yhat;
+  A.G = c->G;
+  A.tab = c->tab;
+  A.dbg_lr = c->dbg_lr;
+  A.dbg_lu = c->dbg_lu;
+  A.acc_len = c->acc_len;
+  const int threads = (A.nq >= 256 || window > 4) ? 256 : 64;
+  verify_kernel<<<c->n, threads, 0, c->stream>>>(A);
+  c->launches++;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Closed-form posterior means (Eq. 4), one warp (mixture) or one block (Gaussian) per point.
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(128) gmm_kernel(RowSet rs, int d, GmmParams P, const float* __restrict__ tt,
+                                                  float* __restrict__ out) {
+  extern __shared__ float s_logit[];  // [warps][n_comp]
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, wpb = blockDim.x >> 5;
+  float* lg = s_logit + warp * P.n_comp;
+  const int n_rows = *rs.n_rows_dev;
+  for (int r = blockIdx.x * wpb + warp; r < n_rows; r += gridDim.x * wpb) {
+    const float* y = rs.ysrc + (size_t)(rs.row_map ? rs.row_map[r] : r) * d;
+    const float t = tt[rs.row_step[r]];
+    const float inv_den = 1.f / (1.f + t * P.s2);
+    float mx = -INFINITY;
+    for (int c = 0; c < P.n_comp; ++c) {
+      float dot = 0.f;
+      for (int k = lane; k < d; k += 32) dot = fmaf(y[k], P.means[(size_t)c * d + k], dot);
+      dot = warp_sum(dot);
+      const float l = P.log_pi[c] + (dot - 0.5f * t * P.cnorm[c]) * inv_den;
+      if (lane == 0) lg[c] = l;
+      mx = fmaxf(mx, l);
+    }
+    __syncwarp();
+    float sum = 0.f;
+    for (int c = 0; c < P.n_comp; ++c) sum += expf(lg[c] - mx);
+    const float inv_sum = 1.f / sum;
+    for (int k = lane; k < d; k += 32) {
+      float acc = 0.f;
+      for (int c = 0; c < P.n_comp; ++c) acc = fmaf(expf(lg[c] - mx) * inv_sum, P.means[(size_t)c * d + k], acc);
+      out[(size_t)r * d + k] = (acc + P.s2 * y[k]) * inv_den;
+    }
+    __syncwarp();
+  }
+}
+
+void launch_gmm(Ctx* c, const RowSet& rs, float* out) {
+  if (rs.n_rows_max <= 0) return;
+  const int threads = 128, wpb = threads / 32;
+  int blocks = (rs.n_rows_max + wpb - 1) / wpb;
+  blocks = blocks > 8 * c->num_sms ? 8 * c->num_sms : blocks;
+  gmm_kernel<<<blocks, threads, wpb * c->gmm.n_comp * sizeof(float), c->stream>>>(rs, c->d, c->gmm, c->tab.tt, out);
+  c->launches++;
+}
+
+__global__ void __launch_bounds__(128) gauss_kernel(RowSet rs, int d, GaussParams P, const float* __restrict__ tt,
+                                                    float* __restrict__ out) {
+  extern __shared__ float s_buf[];  // y[d], w[d]
+  float* ys = s_buf;
+  float* ws = s_buf + d;
+  const int n_rows = *rs.n_rows_dev;
+  for (int r = blockIdx.x; r < n_rows; r += gridDim.x) {
+    const float* y = rs.ysrc + (size_t)(rs.row_map ? rs.row_map[r] : r) * d;
+    const float t = tt[rs.row_step[r]];
+    for (int k = threadIdx.x; k < d; k += blockDim.x) ys[k] = y[k];
+    __syncthreads();
+    for (int jj = threadIdx.x; jj < d; jj += blockDim.x) {
+      float z = 0.f;  // (Q^T y)_j
+      for (int i = 0; i < d; ++i) z = fmaf(P.Q[(size_t)i * d + jj], ys[i], z);
+      const float lam = P.lam[jj];
+      ws[jj] = (P.qmu[jj] + lam * z) / (1.f + t * lam);
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < d; i += blockDim.x) {
+      float m = 0.f;
+      for (int jj = 0; jj < d; ++jj) m = fmaf(P.Qt[(size_t)jj * d + i], ws[jj], m);
+      out[(size_t)r * d + i] = m;
+    }
+    __syncthreads();
+  }
+}
+
+void launch_gauss(Ctx* c, const RowSet& rs, float* out) {
+  if (rs.n_rows_max <= 0) return;
+  int blocks = rs.n_rows_max > 16 * c->num_sms ? 16 * c->num_sms : rs.n_rows_max;
+  const int threads = c->d >= 128 ? 128 : 64;
+  gauss_kernel<<<blocks, threads, 2 * c->d * sizeof(float), c->stream>>>(rs, c->d, c->gauss, c->tab.tt, out);
+  c->launches++;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Network input rows for an arbitrary row set: [bf16(c_in y) ; cond ; temb ; 0].
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) pack_kernel(RowSet rs, int d, MlpParams M, const float* __restrict__ c_in) {
+  const int n_rows = *rs.n_rows_dev;
+  for (int r = blockIdx.x; r < n_rows; r += gridDim.x) {
+    const float* y = rs.ysrc + (size_t)(rs.row_map ? rs.row_map[r] : r) * d;
+    const int step = rs.row_step[r];
+    const float ci = c_in[step];
+    __nv_bfloat16* xr = M.X + (size_t)r * M.in_pad;
+    for (int e = threadIdx.x; e < M.in_pad; e += blockDim.x) {
+      __nv_bfloat16 val = __float2bfloat16_rn(0.f);
+      if (e < d)
+        val = __float2bfloat16_rn(ci * y[e]);
+      else if (e < d + M.d_cond)
+        val = M.cond[(size_t)rs.row_slot[r] * M.d_cond + (e - d)];
+      else if (e < M.in_dim)
+        val = M.temb[(size_t)step * M.d_temb + (e - d - M.d_cond)];
+      xr[e] = val;
+    }
+  }
+}
+
+void launch_pack(Ctx* c, const RowSet& rs) {
+  if (rs.n_rows_max <= 0) return;
+  int blocks = rs.n_rows_max > 8 * c->num_sms ? 8 * c->num_sms : rs.n_rows_max;
+  pack_kernel<<<blocks, 256, 0, c->stream>>>(rs, c->d, c->mlp, c->tab.c_in);
+  c->launches++;
+}
+
+__global__ void cond_to_bf16_kernel(const float* __restrict__ src, __nv_bfloat16* __restrict__ dst, size_t n) {
+  for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x)
+    dst[i] = __float2bfloat16_rn(src[i]);
+}
+
+void launch_cond_to_bf16(Ctx* c, int n) {
+  const size_t total = (size_t)n * c->mlp.d_cond;
+  if (total == 0) return;
+  int blocks = (int)((total + 255) / 256);
+  blocks = blocks > 1024 ? 1024 : blocks;
+  cond_to_bf16_kernel<<<blocks, 256, 0, c->stream>>>(c->cond_f32, const_cast<__nv_bfloat16*>(c->mlp.cond), total);
+  c->launches++;
+}
+
+__global__ void fill_int_kernel(int* p, int n, int val) {
+  for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x) p[i] = val;
+}
+
+void launch_fill_int(Ctx* c, int* p, int n, int val) {
+  if (n <= 0) return;
+  int blocks = (n + 255) / 256;
+  blocks = blocks > 1024 ? 1024 : blocks;
+  fill_int_kernel<<<blocks, 256, 0, c->stream>>>(p, n, val);
+  c->launches++;
+}
+
+}  // namespace asd

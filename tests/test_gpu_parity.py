@@ -1,0 +1,221 @@
+"""GPU parity tests proper: the CUDA library (through the C ABI) against the CPU oracle on the
+same seeded inputs.  Tolerances: fp32 states 1e-4 relative L2 (1e-2 for the bf16 network),
+accept decisions identical whenever |ln ratio - ln u| > 1e-3, prefix lengths bit-exact under
+that margin."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import workloads
+from oracle import asd as oasd
+from oracle import denoisers as oden
+from tests._parity import MARGIN, lockstep, oracle_run, rel_l2, tolerances
+
+pytestmark = pytest.mark.gpu
+
+
+def _sampler(wl, **kw):
+    from paper_2505_03983_b200 import AsdSampler
+    return AsdSampler(wl, **kw)
+
+
+def _log(msg):
+    print(msg)
+
+
+# ------------------------------------------------------------------ drift alone
+@pytest.mark.parametrize("name,n_rows", [("cfg1_gmm2d", 100), ("gmm_odd", 57), ("gauss_small", 50),
+                                         ("cfg2_gauss64", 300), ("mlp_tiny", 23), ("mlp_ragged", 300),
+                                         ("mlp_ragged", 1), ("cfg3_policy", 700)])
+def test_drift_matches_oracle(name, n_rows):
+    wl = workloads.make(name)
+    rng = np.random.default_rng(5)
+    chains = wl.chains
+    cap = max(chains, -(-n_rows // max(wl.window - 1, 1)))
+    with _sampler(wl, max_chains=cap) as s:
+        cond = None
+        if wl.kind == "mlp" and wl.d_cond:
+            cond = np.concatenate([wl.cond] * (-(-cap // chains)))[:cap]
+            wl.cond = cond
+        s.reset(cap, 0, cond=cond)
+        steps = rng.integers(0, wl.K, n_rows).astype(np.int32)
+        tt = wl.t[steps]
+        xstar = rng.standard_normal((n_rows, wl.d))
+        y = (tt[:, None] * xstar + np.sqrt(tt)[:, None] * rng.standard_normal((n_rows, wl.d))).astype(np.float32)
+        slots = rng.integers(0, cap, n_rows).astype(np.int32)
+        out = s.denoise(steps, y, slots).cpu().numpy()
+    g = oden.from_workload(wl)
+    tol = 2e-3 if wl.kind == "mlp" else 2e-5
+    worst = 0.0
+    for r in range(n_rows):
+        ref = g(int(steps[r]), y[r].astype(np.float64), int(slots[r]))
+        err = np.max(np.abs(out[r] - ref)) / max(1.0, np.max(np.abs(ref)))
+        worst = max(worst, err)
+    _log(f"drift {name} rows={n_rows}: max scaled error {worst:.3e}")
+    assert worst < tol
+
+
+# ------------------------------------------------------------------ lock-step rounds
+@pytest.mark.parametrize("name,chains,rounds", [
+    ("cfg1_gmm2d", 16, 60), ("gmm_odd", 9, 30), ("gauss_small", 11, 40), ("cfg2_gauss64", 24, 12),
+    ("mlp_tiny", 5, 25), ("mlp_ragged", 37, 8), ("cfg3_policy", 64, 3)])
+def test_lockstep_rounds(name, chains, rounds):
+    wl = workloads.make(name, chains=chains)
+    with _sampler(wl) as s:
+        worst = lockstep(s, wl, chains, rounds, chain_base=1000, cond=wl.cond if wl.kind == "mlp" and wl.d_cond else None,
+                         log=_log)
+    assert worst["decided"] > 0
+
+
+def test_lockstep_window_64_and_window_beyond_K():
+    wl = workloads.make("gauss_small", K=70, window=64, chains=6)
+    with _sampler(wl) as s:
+        lockstep(s, wl, 6, 10, log=_log)
+    wl = workloads.make("cfg1_gmm2d", K=20, window=64, chains=4)     # window > K acts like K
+    with _sampler(wl) as s:
+        assert s.window == 64
+        wl.window = 20
+        s.window = 20
+        lockstep(s, wl, 4, 10, log=_log)
+
+
+# ------------------------------------------------------------------ whole runs
+@pytest.mark.parametrize("name,chains", [("cfg1_gmm2d", 16), ("gauss_small", 11), ("cfg2_gauss64", 16)])
+def test_free_running_matches_oracle(name, chains):
+    wl = workloads.make(name, chains=chains)
+    with _sampler(wl) as s:
+        s.reset(chains, 0)
+        y, rounds, stats = s.sample()
+        y, rounds = y.cpu().numpy(), rounds.cpu().numpy()
+    ref = oracle_run(wl, range(chains))
+    tol_y, _ = tolerances(wl.kind)
+    compared = 0
+    for j, res in enumerate(ref):
+        if res.min_margin > MARGIN:        # every decision of this chain is outside the margin
+            compared += 1
+            assert rounds[j] == res.rounds, (j, rounds[j], res.rounds)
+            assert rel_l2(y[j].astype(np.float64), res.y) < tol_y
+    assert compared >= 3          # a K=1000 chain takes hundreds of decisions; few stay outside the margin throughout
+    assert stats.rounds_max == rounds.max() and stats.rounds_mean == pytest.approx(rounds.mean())
+    assert math.ceil(wl.K / wl.window) <= rounds.min() and rounds.max() <= math.ceil(wl.K / 2)
+    assert stats.launches > 0
+
+
+@pytest.mark.parametrize("name", ["cfg1_gmm2d", "gauss_small", "mlp_tiny"])
+def test_sequential_matches_oracle_and_window_one(name):
+    wl = workloads.make(name)
+    cond = wl.cond if wl.kind == "mlp" and wl.d_cond else None
+    n = wl.chains
+    with _sampler(wl) as s:
+        s.reset(n, 7, cond=cond)
+        y_seq, st = s.sequential_ddpm()
+        y_seq = y_seq.cpu().numpy()
+        assert st.rows_total == n * wl.K
+    with _sampler(wl, window=1) as s1:
+        s1.reset(n, 7, cond=cond)
+        y_w1, r_w1, _ = s1.sample()
+        assert torch.all(r_w1 == wl.K)
+        assert np.array_equal(y_w1.cpu().numpy(), y_seq)          # bit for bit
+    ref = oracle_run(wl, range(7, 7 + n), slots=list(range(n)), sequential=True)
+    tol_y = 5e-2 if wl.kind == "mlp" else 1e-4    # free-running through a random network amplifies rounding
+    for j in range(n):
+        assert rel_l2(y_seq[j].astype(np.float64), ref[j]) < tol_y
+
+
+def test_batch_and_partition_invariance():
+    """A chain's result depends only on its id: alone, inside a batch, or in a shifted partition."""
+    wl = workloads.make("cfg2_gauss64", chains=12, K=200)
+    with _sampler(wl) as s:
+        s.reset(12, 100)
+        y_all, r_all, _ = s.sample()
+        s.reset(5, 104)
+        y_part, r_part, _ = s.sample()
+        s.reset(1, 107)
+        y_one, r_one, _ = s.sample()
+    assert torch.equal(y_all[4:9], y_part) and torch.equal(r_all[4:9], r_part)
+    assert torch.equal(y_all[7:8], y_one) and torch.equal(r_all[7:8], r_one)
+
+
+def test_state_save_restore_and_y0():
+    wl = workloads.make("gauss_small", chains=8)
+    with _sampler(wl) as s:
+        s.reset(8, 3)
+        y_ref, r_ref, _ = s.sample()
+        s.reset(8, 3)
+        for _ in range(5):
+            s.round(want_stats=False)
+        a, y, r = s.get_state()
+    with _sampler(wl) as s2:
+        s2.reset(8, 3)
+        s2.set_state(a, y, r)
+        y2, r2, _ = s2.sample()
+    assert torch.equal(y2, y_ref) and torch.equal(r2, r_ref)
+    # a non-zero starting point is honoured
+    with _sampler(wl) as s3:
+        y0 = torch.full((8, wl.d), 0.25, device="cuda")
+        s3.reset(8, 3, y0=y0)
+        s3.round()
+        a3, y3, _ = s3.get_state()
+    g, sch = oden.from_workload(wl), oasd.make_schedule(wl.t)
+    rec = oasd.asd_round(g, sch, wl.seed, 3, 0, 0, np.full(wl.d, 0.25), wl.window)
+    assert int(a3[0]) == rec.a_after and rel_l2(y3[0].cpu().numpy().astype(np.float64), rec.y_after) < 1e-4
+
+
+def test_host_buffer_entry_point():
+    wl = workloads.make("cfg1_gmm2d")
+    with _sampler(wl) as s:
+        s.reset(16, 0)
+        y_dev, r_dev, _ = s.sample()
+        y_h, r_h, st = s.sample_host(16, 0)
+        assert np.array_equal(y_h, y_dev.cpu().numpy()) and np.array_equal(r_h, r_dev.cpu().numpy())
+        y_s, _, _ = s.sample_host(16, 0, sequential=True)
+        s.reset(16, 0)
+        y_sd, _ = s.sequential_ddpm()
+        assert np.array_equal(y_s, y_sd.cpu().numpy())
+
+
+def test_empty_and_degenerate_inputs():
+    from paper_2505_03983_b200 import AsdError
+    wl = workloads.make("cfg1_gmm2d", K=1, window=1, chains=3)
+    with _sampler(wl) as s:
+        s.reset(0)
+        y, r, st = s.sample()
+        assert y.shape == (0, 2) and st.rounds_max == 0
+        s.reset(3)
+        y, r, _ = s.sample()
+        assert torch.all(r == 1)
+        with pytest.raises(AsdError):
+            s.reset(4)                                   # beyond max_chains
+    with pytest.raises(AsdError):
+        _sampler(wl, window=0)
+    with pytest.raises(AsdError):
+        _sampler(wl, window=65)
+    bad = workloads.make("cfg1_gmm2d")
+    bad.t = bad.t[::-1].copy()
+    with pytest.raises(AsdError):
+        _sampler(bad)
+
+
+def test_gaussian_target_moments_many_chains():
+    """cfg-2 statistical check on the GPU: 16384 ASD chains and 16384 sequential chains against the
+    closed-form law of the Euler chain (mean T mu0, eigen-variances (1+T lam)^2 sum eta/(1+t lam)^2)."""
+    n = 16384
+    wl = workloads.make("cfg2_gauss64", chains=n, K=250)
+    Q, lam, mu0 = wl.Q.astype(np.float64), wl.lam.astype(np.float64), wl.mu0.astype(np.float64)
+    T = wl.t[-1]
+    eta = np.diff(wl.t)
+    var = (1 + T * lam) ** 2 * np.sum(eta[:, None] / (1 + wl.t[1:, None] * lam[None, :]) ** 2, axis=0)
+    with _sampler(wl) as s:
+        s.reset(n, 0)
+        ya, rounds, st = s.sample()
+        s.reset(n, n)
+        ys, _ = s.sequential_ddpm()
+    _log(f"cfg2 K=250 n={n}: rounds mean {st.rounds_mean:.1f} max {st.rounds_max}")
+    for ysamp in (ya.cpu().numpy().astype(np.float64), ys.cpu().numpy().astype(np.float64)):
+        z = (ysamp - T * mu0) @ Q                   # eigen-coordinates, independent with variance `var`
+        assert np.all(np.abs(z.mean(0)) < 4.5 * np.sqrt(var / n))
+        assert np.all(np.abs(z.var(0, ddof=1) - var) < 4.5 * var * math.sqrt(2 / (n - 1)))
+        C = np.corrcoef(z.T)
+        assert np.max(np.abs(C - np.eye(wl.d))) < 5.5 / math.sqrt(n)
