@@ -1,0 +1,301 @@
+#!/usr/bin/env python
+"""Benchmark of the ASD hot path on B200.
+
+A "step" is one pass of the whole hot path over one batch: reset the chains and run speculation
+rounds (drift at the current points, draft, batched drift at the drafted points, verify,
+advance) until every chain has reached step K.  The metric is samples per second.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
+
+Under torchrun (N > 1) every rank runs the same number of chains with its own chain ids
+(weak scaling, no data-path collective); `value` is all ranks' samples over the max time.
+`--impl reference` times the CPU oracle on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import workloads  # noqa: E402
+
+DEFAULT_WORKLOAD = "sweep_b512_w64"   # cfg-4 denoiser, 512 chains x window 64, K = 1000 (largest cell)
+METRIC = "samples_per_sec"
+UNIT = "samples/s"
+
+
+def read_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return dict(hbm_gbs=p["hbm_gbs"], bf16_tflops=p["bf16_tflops"],
+                    bf16_tflops_sustained=p.get("bf16_tflops_sustained", p["bf16_tflops"]), source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            threading.Thread(target=self._read, daemon=True).start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=["nvidia-smi unavailable"])
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            if len(r) < 6:
+                continue
+            try:
+                sm.append(float(r[0])); mx.append(float(r[1]))
+            except ValueError:
+                continue
+            for nm, val in zip(names, r[2:6]):
+                if val.lower().startswith("active"):
+                    reasons.add(nm)
+        return dict(sm_mhz=float(np.median(sm)) if sm else None, sm_max_mhz=max(mx) if mx else None,
+                    reasons=sorted(reasons), samples=len(sm))
+
+
+def oracle_sample_rate(wl, budget_s: float, max_rounds: int):
+    """Runs the oracle's ASD on chain 0 for at most `max_rounds` rounds / `budget_s` seconds and
+    returns (samples per second extrapolated by the fraction of the K steps covered, description)."""
+    from oracle import asd as oasd, denoisers as oden
+    g = oden.from_workload(wl)
+    sch = oasd.make_schedule(wl.t)
+    y, a, rounds = np.zeros(wl.d), 0, 0
+    t0 = time.perf_counter()
+    while a < wl.K and rounds < max_rounds and time.perf_counter() - t0 < budget_s:
+        rec = oasd.asd_round(g, sch, wl.seed, 0, 0, a, y, wl.window)
+        a, y, rounds = rec.a_after, rec.y_after, rounds + 1
+    el = time.perf_counter() - t0
+    frac = a / wl.K
+    return frac / el, f"chain 0, first {rounds} rounds ({a} of {wl.K} steps) in {el:.1f} s, extrapolated by steps"
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    wl = workloads.make(args.workload)
+    try:
+        import threadpoolctl
+        cores = max(int(i.get("num_threads", 1)) for i in threadpoolctl.threadpool_info()) if threadpoolctl.threadpool_info() else 1
+    except Exception:
+        cores = os.cpu_count() or 1
+    for _ in range(args.warmup):
+        oracle_sample_rate(wl, 2.0, 1)
+    t0 = time.perf_counter()
+    rates, desc = [], ""
+    for _ in range(args.steps):
+        r, desc = oracle_sample_rate(wl, 10.0, 3)
+        rates.append(r)
+    el = time.perf_counter() - t0
+    value = float(np.mean(rates))
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * el / max(args.steps, 1),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": wl.name, "chains": wl.chains, "K": wl.K, "window": wl.window, "d": wl.d},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
+                         "sample": "each step: " + desc},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+def run_ours(args):
+    import torch
+    from paper_2505_03983_b200 import AsdSampler
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    wl = workloads.make(args.workload)
+    n = wl.chains
+    base = rank * n                      # each rank owns its own chain ids: partition-invariant results
+    cond = wl.cond if wl.kind == "mlp" and wl.d_cond else None
+    peaks = read_peaks()
+    s = AsdSampler(wl)
+    cond_dev = None if cond is None else torch.as_tensor(cond, device="cuda")
+
+    def step():
+        s.reset(n, base, cond=cond_dev)
+        return s.sample()
+
+    for _ in range(max(args.warmup, 0)):
+        step()
+    # ---- timed region: device-resident inputs ------------------------------------------------
+    s.set_profiling(True)
+    clocks = ClockSampler(local)
+    barrier()
+    clocks.start()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    launches, rounds_mean, rounds_max, rows = 0, [], [], 0
+    ev0.record()
+    for _ in range(args.steps):
+        y, r, st = step()
+        launches += st.launches
+        rounds_mean.append(st.rounds_mean); rounds_max.append(st.rounds_max); rows += st.rows_total
+    ev1.record()
+    barrier()
+    clk = clocks.stop()
+    ms = ev0.elapsed_time(ev1)
+    prof = s.get_profile()
+    s.set_profiling(False)
+    # ---- end to end through the host-buffer entry point -------------------------------------------
+    y0_h = torch.zeros((n, wl.d), dtype=torch.float32).pin_memory().numpy()
+    cond_h = None if cond is None else torch.as_tensor(cond).pin_memory().numpy()
+    y_h = torch.empty((n, wl.d), dtype=torch.float32).pin_memory().numpy()
+    r_h = torch.zeros((n,), dtype=torch.int32).pin_memory().numpy()
+    s.sample_host(n, base, y0_h, cond_h, False, y_h, r_h)
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        s.sample_host(n, base, y0_h, cond_h, False, y_h, r_h)
+    e1.record()
+    barrier()
+    ms_e2e = e0.elapsed_time(e1)
+    # ---- sequential DDPM (Eq. 7) on the same GPU, one run -------------------------------------------
+    s.reset(n, base, cond=cond_dev)
+    _, st_seq = s.sequential_ddpm()
+    s.close()
+
+    t = torch.tensor([ms, ms_e2e, st_seq.ms_total], dtype=torch.float64, device="cuda")
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms, ms_e2e, ms_seq = [float(x) for x in t.cpu()]
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    total = n * world * args.steps
+    value = total / (ms / 1e3)
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16" if wl.kind == "mlp" else "f32", "data": "synthetic",
+        "config": {"workload": wl.name, "chains_per_gpu": n, "K": wl.K, "window": wl.window, "d": wl.d,
+                   "denoiser": wl.kind, "width": wl.width, "layers": wl.n_layers,
+                   "l2": "working set (weights + activations) larger than L2, no flush needed"
+                         if wl.kind == "mlp" and wl.width >= 4096 else "small working set; L2-resident by design"},
+        "rounds_per_sample": float(np.mean(rounds_mean)), "rounds_max": int(max(rounds_max)),
+        "K_over_rounds": wl.K / float(np.mean(rounds_mean)),
+        "drift_rows_per_sample_over_K": rows / (args.steps * n * wl.K),
+        "gpu_launches": int(launches),
+        "clocks": clk,
+        "e2e": {"value": total / (ms_e2e / 1e3), "unit": UNIT,
+                "h2d_bytes_per_step": int(y0_h.nbytes + (0 if cond_h is None else cond_h.nbytes)),
+                "d2h_bytes_per_step": int(y_h.nbytes + r_h.nbytes)},
+        "sequential_gpu": {"value": n * world / (ms_seq / 1e3), "unit": UNIT, "ms": ms_seq,
+                           "wallclock_speedup_asd": (ms_seq) / (ms / args.steps)},
+        "phases_ms": {k: round(v["ms"], 3) for k, v in prof.items() if v["launches"]},
+    }
+    # ---- roofline of the dominant kernel ----------------------------------------------------
+    if wl.kind == "mlp":
+        hid = prof["pass2_gemm_hidden"]
+        flops = 2.0 * wl.width * wl.width * hid["rows"] * wl.n_layers       # all hidden-layer launches of pass 2
+        ach = flops / (hid["ms"] / 1e3) / 1e12 if hid["ms"] > 0 else 0.0
+        peak = peaks["bf16_tflops_sustained"]
+        line["roofline"] = {"kernel": "gemm_kernel<BN,EPI_HID> (pass 2 hidden layers)", "bound": "tensor",
+                            "achieved": ach, "peak": peak, "unit": "TFLOP/s", "frac": ach / peak,
+                            "peak_source": peaks["source"] + " (sustained cuBLAS bf16)",
+                            "frac_of_burst_peak": ach / peaks["bf16_tflops"],
+                            "launches": hid["launches"], "avg_launch_ms": hid["ms"] / max(hid["launches"], 1),
+                            "traffic": None}
+        ver = prof["verify"]
+        # algorithmic bytes of verify: read G once (4 d (w-1) per chain-round = 4 d per pass-2 row),
+        # read y and v, write y (3 * 4 d per chain-round)
+        vbytes = 4.0 * wl.d * (prof["pass2_gemm_out"]["rows"] + 3 * ver["rows"])
+        vach = vbytes / (ver["ms"] / 1e3) / 1e9 if ver["ms"] > 0 else 0.0
+        line["roofline_verify"] = {"kernel": "verify_kernel", "bound": "hbm", "achieved": vach, "peak": peaks["hbm_gbs"],
+                                   "unit": "GB/s", "frac": vach / peaks["hbm_gbs"], "peak_source": peaks["source"],
+                                   "launches": ver["launches"], "avg_launch_ms": ver["ms"] / max(ver["launches"], 1),
+                                   "traffic": None}
+    else:
+        ver = prof["verify"]
+        rows2 = prof["pass2_closed_form"]["rows"]
+        vbytes = 4.0 * wl.d * (rows2 + 3 * ver["rows"])
+        vach = vbytes / (ver["ms"] / 1e3) / 1e9 if ver["ms"] > 0 else 0.0
+        line["roofline"] = {"kernel": "verify_kernel", "bound": "hbm", "achieved": vach, "peak": peaks["hbm_gbs"],
+                            "unit": "GB/s", "frac": vach / peaks["hbm_gbs"], "peak_source": peaks["source"],
+                            "launches": ver["launches"], "avg_launch_ms": ver["ms"] / max(ver["launches"], 1),
+                            "traffic": None}
+    # ---- CPU oracle on a bounded sample (rank 0, N = 1 only) -----------------------------------
+    if world == 1 and not args.no_cpu_baseline:
+        rate, desc = oracle_sample_rate(wl, 20.0, 6 if wl.kind == "mlp" and wl.width >= 4096 else 10 ** 9)
+        try:
+            import threadpoolctl
+            info = threadpoolctl.threadpool_info()
+            cores = max(int(i.get("num_threads", 1)) for i in info) if info else 1
+        except Exception:
+            cores = os.cpu_count() or 1
+        line["cpu_baseline"] = {"value": rate, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc}
+    print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=3)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

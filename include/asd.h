@@ -208,6 +208,23 @@ asd_status asd_debug_last_round(asd_ctx* ctx, float* ln_ratio_dev, float* ln_u_d
 asd_status asd_denoise(asd_ctx* ctx, int32_t n_rows, const int32_t* step_dev, const float* y_dev,
                        const int32_t* slot_dev, float* out_dev);
 
+/*
+ * Measurement aid (the paper has no counterpart): per-phase device time of asd_sample, taken
+ * with CUDA event pairs on the context's stream around the launches of each phase, so a
+ * phase's time is the time its kernels occupied the stream.  asd_set_profiling(ctx, 1) clears
+ * the accumulators and turns the events on (two event records per phase and round);
+ * asd_get_profile copies up to `capacity` entries (name has static storage; launches = kernels
+ * launched in the phase; rows = chains or points processed by it, counted by asd_sample only).
+ */
+typedef struct {
+  const char* name;
+  int64_t launches;
+  double ms;
+  int64_t rows;
+} asd_phase_time;
+asd_status asd_set_profiling(asd_ctx* ctx, int32_t enable);
+asd_status asd_get_profile(asd_ctx* ctx, asd_phase_time* out, int32_t capacity, int32_t* n_out);
+
 /* Message for the last error on this context (static or context storage; never NULL). */
 const char* asd_last_error(const asd_ctx* ctx);
 

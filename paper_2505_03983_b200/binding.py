@@ -16,7 +16,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 EXPORTED_SYMBOLS = [
     "asd_version", "asd_create", "asd_reset", "asd_round", "asd_sample", "asd_sequential_ddpm",
     "asd_sample_host", "asd_get_state", "asd_set_state", "asd_debug_last_round", "asd_denoise",
-    "asd_last_error", "asd_destroy",
+    "asd_set_profiling", "asd_get_profile", "asd_last_error", "asd_destroy",
 ]
 
 STATUS = {0: "ASD_OK", 1: "ASD_ERR_INVALID_ARG", 2: "ASD_ERR_UNSUPPORTED", 3: "ASD_ERR_OOM",
@@ -57,6 +57,10 @@ class _RoundStats(C.Structure):
 class _RunStats(C.Structure):
     _fields_ = [("rounds_max", C.c_int64), ("rounds_mean", C.c_double), ("rows_total", C.c_int64),
                 ("ms_total", C.c_double), ("launches", C.c_int64)]
+
+
+class _PhaseTime(C.Structure):
+    _fields_ = [("name", C.c_char_p), ("launches", C.c_int64), ("ms", C.c_double), ("rows", C.c_int64)]
 
 
 @dataclasses.dataclass
@@ -112,6 +116,8 @@ def load_library():
         "asd_set_state": [vp, vp, vp, vp],
         "asd_debug_last_round": [vp, vp, vp, vp],
         "asd_denoise": [vp, i32, vp, vp, vp, vp],
+        "asd_set_profiling": [vp, i32],
+        "asd_get_profile": [vp, C.POINTER(_PhaseTime), i32, C.POINTER(i32)],
     }
     for name, args in protos.items():
         fn = getattr(lib, name)
@@ -299,3 +305,14 @@ class AsdSampler:
         self._check(self.lib.asd_denoise(self._ctx, y.shape[0], _dev_ptr(steps), _dev_ptr(y), _dev_ptr(slots),
                                          _dev_ptr(out)))
         return out
+
+    def set_profiling(self, enable: bool):
+        self._check(self.lib.asd_set_profiling(self._ctx, int(enable)))
+
+    def get_profile(self):
+        """{phase name: dict(launches, ms, rows)} accumulated since set_profiling(True)."""
+        arr = (_PhaseTime * 32)()
+        n = C.c_int32(0)
+        self._check(self.lib.asd_get_profile(self._ctx, arr, 32, C.byref(n)))
+        return {arr[i].name.decode(): dict(launches=arr[i].launches, ms=arr[i].ms, rows=arr[i].rows)
+                for i in range(n.value)}

@@ -68,6 +68,7 @@ asd_status check_device_error(Ctx* c) {
 asd_status sync_counters(Ctx* c) {
   ASD_CUDA(c, cudaMemcpyAsync(c->counters_host, c->counters, sizeof(RoundCounters), cudaMemcpyDeviceToHost, c->stream));
   ASD_CUDA(c, cudaStreamSynchronize(c->stream));
+  prof_collect(c);
   return check_device_error(c);
 }
 
@@ -75,34 +76,97 @@ asd_status sync_counters(Ctx* c) {
 // one step of Eq. 7).  active_bound: host-side upper bound on the number of active chains.
 asd_status enqueue_round(Ctx* c, int window, bool use_u, int active_bound) {
   if (active_bound <= 0) return ASD_OK;
-  launch_prep(c, window);
+  {
+    ProfScope ps(c, PH_PREP);
+    launch_prep(c, window);
+  }
   RowSet rs1{&c->counters->n_active, active_bound, c->y, c->act, c->step1, c->act};
   RowSet rs2{&c->counters->rows2, active_bound * (window - 1), c->Yhat, nullptr, c->row_step, c->row_slot};
   asd_status st = ASD_OK;
   switch (c->kind) {
     case ASD_DEN_GMM_ISO:
-      launch_gmm(c, rs1, c->v);
-      launch_draft(c, window);
-      launch_gmm(c, rs2, c->G);
+    case ASD_DEN_GAUSS_LINEAR: {
+      const bool gmm = c->kind == ASD_DEN_GMM_ISO;
+      {
+        ProfScope ps(c, PH_D1_ANALYTIC);
+        gmm ? launch_gmm(c, rs1, c->v) : launch_gauss(c, rs1, c->v);
+      }
+      {
+        ProfScope ps(c, PH_DRAFT);
+        launch_draft(c, window);
+      }
+      {
+        ProfScope ps(c, PH_D2_ANALYTIC);
+        gmm ? launch_gmm(c, rs2, c->G) : launch_gauss(c, rs2, c->G);
+      }
       break;
-    case ASD_DEN_GAUSS_LINEAR:
-      launch_gauss(c, rs1, c->v);
-      launch_draft(c, window);
-      launch_gauss(c, rs2, c->G);
-      break;
-    default:
-      launch_pack(c, rs1);
-      st = mlp_forward(c, rs1, c->v);
+    }
+    default: {
+      {
+        ProfScope ps(c, PH_PACK);
+        launch_pack(c, rs1);
+      }
+      st = mlp_forward(c, rs1, c->v, 0);
       if (st != ASD_OK) return st;
-      launch_draft(c, window);
-      st = mlp_forward(c, rs2, c->G);
+      {
+        ProfScope ps(c, PH_DRAFT);
+        launch_draft(c, window);
+      }
+      st = mlp_forward(c, rs2, c->G, 1);
       if (st != ASD_OK) return st;
       break;
+    }
   }
-  launch_verify(c, window, use_u);
+  {
+    ProfScope ps(c, PH_VERIFY);
+    launch_verify(c, window, use_u);
+  }
   ASD_CUDA(c, cudaGetLastError());
   return ASD_OK;
 }
+
+}  // namespace
+
+namespace asd {
+ProfScope::ProfScope(Ctx* c_, int phase_) : c(c_ && c_->prof_on ? c_ : nullptr), phase(phase_), l0(0), e0(0) {
+  if (!c) return;
+  if (c->ev_used + 2 > c->ev_pool.size()) {
+    for (int i = 0; i < 64; ++i) {
+      cudaEvent_t e;
+      if (cudaEventCreate(&e) != cudaSuccess) {
+        c = nullptr;
+        return;
+      }
+      c->ev_pool.push_back(e);
+    }
+  }
+  l0 = c->launches;
+  e0 = c->ev_used;
+  c->ev_used += 2;
+  cudaEventRecord(c->ev_pool[e0], c->stream);
+}
+ProfScope::~ProfScope() {
+  if (!c) return;
+  cudaEventRecord(c->ev_pool[e0 + 1], c->stream);
+  c->pending.push_back({phase, e0, e0 + 1, (int)(c->launches - l0)});
+  c = nullptr;
+}
+void prof_collect(Ctx* c) {
+  if (!c->prof_on && c->pending.empty()) return;
+  for (const auto& p : c->pending) {
+    if (p.launches == 0) continue;
+    float ms = 0.f;
+    if (cudaEventElapsedTime(&ms, c->ev_pool[p.e0], c->ev_pool[p.e1]) == cudaSuccess) {
+      c->prof[p.phase].ms += ms;
+      c->prof[p.phase].launches += p.launches;
+    }
+  }
+  c->pending.clear();
+  c->ev_used = 0;
+}
+}  // namespace asd
+
+namespace {
 
 struct HostTables {
   std::vector<float> eta, sig, c1, c2, tt;
@@ -135,6 +199,7 @@ void asd_destroy(asd_ctx* ctx) {
   if (c->counters_host) cudaFreeHost(c->counters_host);
   if (c->ev0) cudaEventDestroy(c->ev0);
   if (c->ev1) cudaEventDestroy(c->ev1);
+  for (cudaEvent_t e : c->ev_pool) cudaEventDestroy(e);
   delete ctx;
 }
 
@@ -444,6 +509,12 @@ asd_status asd_sample(asd_ctx* ctx, float* y_out_dev, int32_t* rounds_out_dev, a
     st = sync_counters(c);
     if (st != ASD_OK) return st;
     active = c->counters_host->n_active_after;
+    if (c->prof_on) {
+      const long long n1 = c->counters_host->n_active, n2 = c->counters_host->rows2;
+      for (int ph : {PH_PREP, PH_PACK, PH_D1_IN, PH_D1_HID, PH_D1_OUT, PH_D1_ANALYTIC, PH_DRAFT, PH_VERIFY})
+        c->prof[ph].rows += n1;
+      for (int ph : {PH_D2_IN, PH_D2_HID, PH_D2_OUT, PH_D2_ANALYTIC}) c->prof[ph].rows += n2;
+    }
   }
   if (active > 0) return fail(c, ASD_ERR_STATE, "chains still active after K rounds");
   return finish_run(c, y_out_dev, rounds_out_dev, stats_host, launches0, true);
@@ -503,6 +574,34 @@ asd_status asd_sample_host(asd_ctx* ctx, int32_t n_chains, uint64_t chain_id_bas
   return ASD_OK;
 }
 
+asd_status asd_set_profiling(asd_ctx* ctx, int32_t enable) {
+  if (!ctx) return ASD_ERR_INVALID_ARG;
+  Ctx* c = &ctx->c;
+  cudaStreamSynchronize(c->stream);
+  prof_collect(c);
+  c->prof_on = enable != 0;
+  for (auto& p : c->prof) p = PhaseAcc{};
+  return ASD_OK;
+}
+
+asd_status asd_get_profile(asd_ctx* ctx, asd_phase_time* out, int32_t capacity, int32_t* n_out) {
+  if (!ctx || !out || !n_out) return ASD_ERR_INVALID_ARG;
+  Ctx* c = &ctx->c;
+  static const char* names[PH_COUNT] = {"prep", "pack", "pass1_gemm_in", "pass1_gemm_hidden", "pass1_gemm_out",
+                                        "pass1_closed_form", "draft", "pass2_gemm_in", "pass2_gemm_hidden",
+                                        "pass2_gemm_out", "pass2_closed_form", "verify"};
+  int k = 0;
+  for (int ph = 0; ph < PH_COUNT && k < capacity; ++ph) {
+    out[k].name = names[ph];
+    out[k].launches = c->prof[ph].launches;
+    out[k].ms = c->prof[ph].ms;
+    out[k].rows = c->prof[ph].rows;
+    ++k;
+  }
+  *n_out = k;
+  return ASD_OK;
+}
+
 asd_status asd_get_state(asd_ctx* ctx, int32_t* a_dev, float* y_dev, int32_t* rounds_dev) {
   if (!ctx) return ASD_ERR_INVALID_ARG;
   Ctx* c = &ctx->c;
@@ -556,7 +655,7 @@ asd_status asd_denoise(asd_ctx* ctx, int32_t n_rows, const int32_t* step_dev, co
     launch_gauss(c, rs, out_dev);
   else {
     launch_pack(c, rs);
-    st = mlp_forward(c, rs, out_dev);
+    st = mlp_forward(c, rs, out_dev, 2);
     if (st != ASD_OK) return st;
   }
   ASD_CUDA(c, cudaGetLastError());

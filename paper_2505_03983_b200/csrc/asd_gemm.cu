@@ -445,7 +445,7 @@ int pick_bn(const Ctx* c, int m_bound, int n_out) {
 
 }  // namespace
 
-asd_status mlp_forward(Ctx* c, const RowSet& rs, float* out) {
+asd_status mlp_forward(Ctx* c, const RowSet& rs, float* out, int pass) {
   const MlpParams& M = c->mlp;
   const int m_bound = rs.n_rows_max;
   if (m_bound <= 0) return ASD_OK;
@@ -461,8 +461,14 @@ asd_status mlp_forward(Ctx* c, const RowSet& rs, float* out) {
   g.out_bf16 = M.H[0];
   g.ld_h = M.width;
   const int bn_h = pick_bn(c, m_bound, M.width);
-  st = launch_gemm<EPI_IN>(c, bn_h, M.X, M.in_pad, M.W_in, g, m_bound);
+  const int ph_in = pass == 0 ? PH_D1_IN : PH_D2_IN, ph_hid = pass == 0 ? PH_D1_HID : PH_D2_HID,
+            ph_out = pass == 0 ? PH_D1_OUT : PH_D2_OUT;
+  {
+    ProfScope ps(pass < 2 ? c : nullptr, ph_in);
+    st = launch_gemm<EPI_IN>(c, bn_h, M.X, M.in_pad, M.W_in, g, m_bound);
+  }
   if (st != ASD_OK) return st;
+  ProfScope ps_hid(pass < 2 ? c : nullptr, ph_hid);
   // residual layers
   for (int l = 0; l < M.n_layers; ++l) {
     g.k_dim = M.width;
@@ -472,6 +478,8 @@ asd_status mlp_forward(Ctx* c, const RowSet& rs, float* out) {
     st = launch_gemm<EPI_HID>(c, bn_h, M.H[l & 1], M.width, M.W_hid + (size_t)l * M.width * M.width, g, m_bound);
     if (st != ASD_OK) return st;
   }
+  ps_hid.~ProfScope();
+  ps_hid.c = nullptr;
   // output projection with the skip / scale epilogue
   g.n_out = c->d;
   g.k_dim = M.width;
@@ -485,6 +493,7 @@ asd_status mlp_forward(Ctx* c, const RowSet& rs, float* out) {
   g.c_skip = c->tab.c_skip;
   g.c_out = c->tab.c_out;
   const int bn_o = pick_bn(c, m_bound, c->d);
+  ProfScope ps_out(pass < 2 ? c : nullptr, ph_out);
   return launch_gemm<EPI_OUT>(c, bn_o, M.H[M.n_layers & 1], M.width, M.W_out, g, m_bound);
 }
 

@@ -83,6 +83,18 @@ struct MlpParams {
   int row_cap;
 };
 
+// Phases of a round, for the optional per-phase CUDA-event timing.
+enum Phase {
+  PH_PREP = 0, PH_PACK, PH_D1_IN, PH_D1_HID, PH_D1_OUT, PH_D1_ANALYTIC, PH_DRAFT,
+  PH_D2_IN, PH_D2_HID, PH_D2_OUT, PH_D2_ANALYTIC, PH_VERIFY, PH_COUNT
+};
+
+struct PhaseAcc {
+  long long launches = 0;
+  double ms = 0.0;
+  long long rows = 0;  // rows (points, chains) processed by the phase
+};
+
 struct Ctx {
   // configuration
   int d = 0, K = 0, window = 0, max_chains = 0, kind = 0;
@@ -122,7 +134,25 @@ struct Ctx {
   std::string err;
   long long launches = 0;
   cudaEvent_t ev0 = nullptr, ev1 = nullptr;
+  // per-phase timing (off by default)
+  bool prof_on = false;
+  PhaseAcc prof[PH_COUNT];
+  std::vector<cudaEvent_t> ev_pool;
+  size_t ev_used = 0;
+  struct Pending { int phase; size_t e0, e1; int launches; };
+  std::vector<Pending> pending;
 };
+
+// Brackets the launches of one phase with two events when timing is on.
+struct ProfScope {
+  Ctx* c;
+  int phase;
+  long long l0;
+  size_t e0;
+  ProfScope(Ctx* c_, int phase_);
+  ~ProfScope();
+};
+void prof_collect(Ctx* c);  // after a stream synchronisation: fold pending event pairs into c->prof
 
 // ---- launchers (asd_kernels.cu) ---------------------------------------------------------
 void launch_prep(Ctx* c, int window);
@@ -136,6 +166,7 @@ void launch_fill_int(Ctx* c, int* p, int n, int val);
 
 // ---- MLP forward (asd_gemm.cu) ----------------------------------------------------------
 // Runs the GEMM chain on the rows already packed into mlp.X; writes out[r] for r < *n_rows_dev.
-asd_status mlp_forward(Ctx* c, const RowSet& rs, float* out);
+// pass: 0 = drift at the current points, 1 = drift at the drafted points, 2 = stand-alone call.
+asd_status mlp_forward(Ctx* c, const RowSet& rs, float* out, int pass);
 
 }  // namespace asd
