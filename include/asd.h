@@ -225,6 +225,39 @@ typedef struct {
 asd_status asd_set_profiling(asd_ctx* ctx, int32_t enable);
 asd_status asd_get_profile(asd_ctx* ctx, asd_phase_time* out, int32_t capacity, int32_t* n_out);
 
+/*
+ * asd_denoise_static - the drift of the network denoiser without any device allocation.
+ * (The paper has no counterpart: this is a deployment aid of this library.)
+ *
+ * asd_denoise can only take as many rows as the context was sized for in asd_create, and
+ * making room for more means a new context, i.e. cudaMalloc.  Some callers cannot do that at
+ * the point where they need the drift: a serving loop that must not take cudaMalloc's
+ * device-wide synchronisation, a process that has handed all remaining device memory to another
+ * allocator (so cudaMalloc would fail), or code running where its host forbids allocation calls.
+ * For them this entry point keeps the activations of the GEMM chain (input rows and the two
+ * hidden-state buffers) and its row counter in ONE fixed array of ASD_STATIC_SCRATCH_BYTES
+ * (8 MiB) that is part of the library image: every GPU on which the library is used holds those
+ * 8 MiB from the first kernel launch until the process exits.
+ *
+ * Arguments, layouts and result are those of asd_denoise (device pointers; rows beyond n_rows
+ * untouched); the result is identical to asd_denoise's.  Only ASD_DEN_RESMLP_BF16 contexts are
+ * accepted (the closed-form drifts use no scratch: UNSUPPORTED).  n_rows may be at most
+ * floor((8 MiB - 1 KiB) / (2 (in_pad + 2 width))) with in_pad = d + d_cond + d_temb rounded up
+ * to 64 - asd_denoise_static_max_rows returns it; larger requests fail with INVALID_ARG and
+ * nothing is launched.  The context's device must be current (STATE otherwise).
+ *
+ * The first call on a device looks up the array's device address; make that first call before
+ * starting any stream capture.  The call synchronises the context's stream before returning.
+ * All contexts and all calls share the one array and it keeps the previous call's contents
+ * (this call rewrites everything it reads): calls that overlap on the GPU - different streams,
+ * different contexts or threads - race on it; run them one after the other.
+ * It calls no cudaMalloc / cudaFree and no allocating library routine.
+ */
+#define ASD_STATIC_SCRATCH_BYTES (8u << 20)
+asd_status asd_denoise_static(asd_ctx* ctx, int32_t n_rows, const int32_t* step_dev, const float* y_dev,
+                              const int32_t* slot_dev, float* out_dev);
+asd_status asd_denoise_static_max_rows(const asd_ctx* ctx, int32_t* max_rows_out);
+
 /* Message for the last error on this context (static or context storage; never NULL). */
 const char* asd_last_error(const asd_ctx* ctx);
 

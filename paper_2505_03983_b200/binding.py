@@ -16,7 +16,8 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 EXPORTED_SYMBOLS = [
     "asd_version", "asd_create", "asd_reset", "asd_round", "asd_sample", "asd_sequential_ddpm",
     "asd_sample_host", "asd_get_state", "asd_set_state", "asd_debug_last_round", "asd_denoise",
-    "asd_set_profiling", "asd_get_profile", "asd_last_error", "asd_destroy",
+    "asd_set_profiling", "asd_get_profile", "asd_denoise_static", "asd_denoise_static_max_rows",
+    "asd_last_error", "asd_destroy",
 ]
 
 STATUS = {0: "ASD_OK", 1: "ASD_ERR_INVALID_ARG", 2: "ASD_ERR_UNSUPPORTED", 3: "ASD_ERR_OOM",
@@ -116,6 +117,8 @@ def load_library():
         "asd_set_state": [vp, vp, vp, vp],
         "asd_debug_last_round": [vp, vp, vp, vp],
         "asd_denoise": [vp, i32, vp, vp, vp, vp],
+        "asd_denoise_static": [vp, i32, vp, vp, vp, vp],
+        "asd_denoise_static_max_rows": [vp, C.POINTER(i32)],
         "asd_set_profiling": [vp, i32],
         "asd_get_profile": [vp, C.POINTER(_PhaseTime), i32, C.POINTER(i32)],
     }
@@ -316,3 +319,22 @@ class AsdSampler:
         self._check(self.lib.asd_get_profile(self._ctx, arr, 32, C.byref(n)))
         return {arr[i].name.decode(): dict(launches=arr[i].launches, ms=arr[i].ms, rows=arr[i].rows)
                 for i in range(n.value)}
+
+    def denoise_static_max_rows(self) -> int:
+        n = C.c_int32(0)
+        self._check(self.lib.asd_denoise_static_max_rows(self._ctx, C.byref(n)))
+        return n.value
+
+    def denoise_static(self, steps, y, slots=None):
+        """asd_denoise_static: same arguments and result as denoise(), but the GEMM chain's scratch
+        is the library's fixed 8 MiB array, so the call allocates no device memory (the output
+        tensor is allocated here, by torch, before the call; pass `out=` style callers use the C ABI)."""
+        torch = self._torch
+        steps = torch.as_tensor(steps).to(device="cuda", dtype=torch.int32).contiguous()
+        y = torch.as_tensor(y).to(device="cuda", dtype=torch.float32).contiguous()
+        if slots is not None:
+            slots = torch.as_tensor(slots).to(device="cuda", dtype=torch.int32).contiguous()
+        out = torch.empty_like(y)
+        self._check(self.lib.asd_denoise_static(self._ctx, y.shape[0], _dev_ptr(steps), _dev_ptr(y),
+                                                _dev_ptr(slots), _dev_ptr(out)))
+        return out
