@@ -290,8 +290,23 @@ def main():
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--profile-rounds", type=int, default=0,
+                    help="profiling aid: reset, run this many speculation rounds, print nothing timed and exit "
+                         "(a short, bounded launch sequence for ncu captures)")
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.profile_rounds > 0:
+        import torch
+        from paper_2505_03983_b200 import AsdSampler
+        wl = workloads.make(args.workload)
+        with AsdSampler(wl) as s:
+            cond = torch.as_tensor(wl.cond, device="cuda") if wl.kind == "mlp" and wl.d_cond else None
+            s.reset(wl.chains, 0, cond=cond)
+            for _ in range(args.profile_rounds):
+                st = s.round()
+            print(json.dumps({"profile_rounds": args.profile_rounds, "workload": wl.name,
+                              "last_round": {"active": st.n_active_before, "rows_pass2": st.rows_pass2,
+                                             "accepted": st.accepted_total}}))
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)
