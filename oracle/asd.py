@@ -107,6 +107,8 @@ class RoundRecord:
     ln_u: np.ndarray           # [w]
     y_after: np.ndarray
     new_states: List[np.ndarray]   # y_{a+1} .. y_{a_after}
+    points: Optional[List[np.ndarray]] = None   # diagnostics: y^_a .. y^_{b-1}, where the drift was evaluated
+    drift: Optional[List[np.ndarray]] = None    # diagnostics: g(t_i, y^_i) at those points (drift[0] = v_a)
 
     @property
     def margin(self) -> float:
@@ -156,7 +158,7 @@ def asd_round(g: Callable, sched: Schedule, seed: int, chain_id: int, slot: int,
     else:
         new_states = zs[:n]
         a_after = a + n
-    return RoundRecord(a, w, n, a_after, ln_ratio, ln_u, new_states[-1], new_states)
+    return RoundRecord(a, w, n, a_after, ln_ratio, ln_u, new_states[-1], new_states, y_hat[:w], drift)
 
 
 @dataclasses.dataclass
