@@ -15,6 +15,8 @@
 // ASD_ERR_TIMEOUT in the context's device error word and carries on as if the wait had
 // completed, so the kernel always reaches its tear-down (tensor memory is released) and the host
 // reports the error after the call.
+#include <algorithm>
+
 #include "asd_internal.h"
 
 namespace asd {
@@ -85,6 +87,15 @@ __device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatil
     }
   }
 }
+// After a wait has run out the producer may still have copies in flight into this CTA's shared
+// memory; give them time to land before the CTA exits (error path only).
+__device__ __forceinline__ void drain_after_timeout(volatile int* dead) {
+  if (*dead) {
+    const long long t0 = clock64();
+    while (clock64() - t0 < 2000000ll) {
+    }
+  }
+}
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y) {
   asm volatile(
       "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];" ::"r"(dst),
@@ -120,6 +131,52 @@ __device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&r)[32]) {
 }
 __device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
+// ---- CTA-pair (cta_group::2) variants ------------------------------------------------------------
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+// Address of the same shared-memory location in CTA `rank` of the cluster (shared::cluster window).
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// Arrive on a barrier that may live in the peer CTA (shared::cluster address).
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t bar_cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(bar_cluster_addr) : "memory");
+}
+// TMA load into this CTA's shared memory whose completion bytes are counted on a barrier of either
+// CTA of the pair (no multicast: every CTA fetches its own box).
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, uint32_t bar_cluster_addr, int x,
+                                                 int y) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], "
+      "[%2];" ::"r"(dst),
+      "l"(map), "r"(bar_cluster_addr), "r"(x), "r"(y)
+      : "memory");
+}
+// Commit of the pair's MMAs issued so far: one arrival on the given barrier (shared::cluster address).
+__device__ __forceinline__ void tc_commit_pair(uint32_t bar_cluster_addr) {
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar_cluster_addr)
+               : "memory");
+}
+// D[256 x N] (+)= A[256 x 16] B[N x 16]^T over the CTA pair: each CTA supplies 128 rows of A and N/2
+// rows of B from the same shared-memory offsets and receives its 128 rows of D in its own tensor memory.
+__device__ __forceinline__ void tc_mma_bf16_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                                 uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5, %5, %5, %5, %5}, p;\n\t}" ::"r"(d_tmem),
+      "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(0u)
+      : "memory");
+}
+
 // Shared-memory matrix descriptor of a K-major tile stored as rows of 128 bytes with the 128-byte
 // swizzle (what the TMA writes): start address, leading byte offset 1 (unused for swizzled K-major),
 // stride byte offset 1024 (8 rows x 128 B), descriptor version 1, layout type 2 (128-byte swizzle).
@@ -148,6 +205,77 @@ struct Cfg {
 };
 
 __device__ __forceinline__ float silu(float z) { return z / (1.0f + __expf(-z)); }
+
+// Epilogue of 32 consecutive accumulator columns [col0, col0 + 32) of one output row held by this
+// thread: bias, then the layer's fused tail, then the store (16-byte vectors where the shape allows).
+template <int EPI>
+__device__ __forceinline__ void epilogue_chunk(const GemmArgs& g, int row, int col0, const uint32_t (&r)[32], float cs,
+                                               float co, const float* ysrc_row) {
+  if (EPI == EPI_OUT) {
+    float* orow = g.out_f32 + (size_t)row * g.n_out;
+    const bool vec = (g.n_out % 4 == 0) && (col0 + 32 <= g.n_out);
+    if (vec) {
+#pragma unroll
+      for (int e = 0; e < 32; e += 4) {
+        const float4 b4 = *reinterpret_cast<const float4*>(g.bias + col0 + e);
+        const float4 y4 = *reinterpret_cast<const float4*>(ysrc_row + col0 + e);
+        float4 o;
+        o.x = fmaf(cs, y4.x, co * (__uint_as_float(r[e + 0]) + b4.x));
+        o.y = fmaf(cs, y4.y, co * (__uint_as_float(r[e + 1]) + b4.y));
+        o.z = fmaf(cs, y4.z, co * (__uint_as_float(r[e + 2]) + b4.z));
+        o.w = fmaf(cs, y4.w, co * (__uint_as_float(r[e + 3]) + b4.w));
+        *reinterpret_cast<float4*>(orow + col0 + e) = o;
+      }
+    } else {
+#pragma unroll
+      for (int e = 0; e < 32; ++e) {
+        const int col = col0 + e;
+        if (col < g.n_out)
+          orow[col] = fmaf(cs, ysrc_row[col], co * (__uint_as_float(r[e]) + g.bias[col]));
+      }
+    }
+  } else {
+    __nv_bfloat16* orow = g.out_bf16 + (size_t)row * g.ld_h;
+    const __nv_bfloat16* rrow = (EPI == EPI_HID) ? g.resid + (size_t)row * g.ld_h : nullptr;
+    const bool vec = (g.ld_h % 8 == 0) && (col0 + 32 <= g.n_out);
+    if (vec) {
+#pragma unroll
+      for (int e = 0; e < 32; e += 8) {
+        float x[8];
+        const float4 b0 = *reinterpret_cast<const float4*>(g.bias + col0 + e);
+        const float4 b1 = *reinterpret_cast<const float4*>(g.bias + col0 + e + 4);
+        const float bb[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
+#pragma unroll
+        for (int u = 0; u < 8; ++u) x[u] = __uint_as_float(r[e + u]) + bb[u];
+        if (EPI == EPI_HID) {
+          const uint4 rv = *reinterpret_cast<const uint4*>(rrow + col0 + e);
+          const __nv_bfloat162* rp = reinterpret_cast<const __nv_bfloat162*>(&rv);
+#pragma unroll
+          for (int u = 0; u < 4; ++u) {
+            const float2 rf = __bfloat1622float2(rp[u]);
+            x[2 * u] = rf.x + silu(x[2 * u]);
+            x[2 * u + 1] = rf.y + silu(x[2 * u + 1]);
+          }
+        }
+        uint4 ov;
+        __nv_bfloat162* op = reinterpret_cast<__nv_bfloat162*>(&ov);
+#pragma unroll
+        for (int u = 0; u < 4; ++u) op[u] = __floats2bfloat162_rn(x[2 * u], x[2 * u + 1]);
+        *reinterpret_cast<uint4*>(orow + col0 + e) = ov;
+      }
+    } else {
+#pragma unroll
+      for (int e = 0; e < 32; ++e) {
+        const int col = col0 + e;
+        if (col < g.n_out) {
+          float x = __uint_as_float(r[e]) + g.bias[col];
+          if (EPI == EPI_HID) x = __bfloat162float(rrow[col]) + silu(x);
+          orow[col] = __float2bfloat16_rn(x);
+        }
+      }
+    }
+  }
+}
 
 template <int BN, int EPI>
 __global__ void __launch_bounds__(kGemmThreads, 1)
@@ -216,6 +344,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
           }
         }
       }
+      drain_after_timeout(dead);
     }
   } else if (warp == 1) {
     // ---------------- MMA issuer ----------------
@@ -277,72 +406,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         tc_ld32(taddr, r);
         tc_wait_ld();
         const int col0 = n0 + c0;
-        if (row_ok && col0 < g.n_out) {
-          if (EPI == EPI_OUT) {
-            float* orow = g.out_f32 + (size_t)row * g.n_out;
-            const bool vec = (g.n_out % 4 == 0) && (col0 + 32 <= g.n_out);
-            if (vec) {
-#pragma unroll
-              for (int e = 0; e < 32; e += 4) {
-                const float4 b4 = *reinterpret_cast<const float4*>(g.bias + col0 + e);
-                const float4 y4 = *reinterpret_cast<const float4*>(ysrc_row + col0 + e);
-                float4 o;
-                o.x = fmaf(cs, y4.x, co * (__uint_as_float(r[e + 0]) + b4.x));
-                o.y = fmaf(cs, y4.y, co * (__uint_as_float(r[e + 1]) + b4.y));
-                o.z = fmaf(cs, y4.z, co * (__uint_as_float(r[e + 2]) + b4.z));
-                o.w = fmaf(cs, y4.w, co * (__uint_as_float(r[e + 3]) + b4.w));
-                *reinterpret_cast<float4*>(orow + col0 + e) = o;
-              }
-            } else {
-#pragma unroll
-              for (int e = 0; e < 32; ++e) {
-                const int col = col0 + e;
-                if (col < g.n_out)
-                  orow[col] = fmaf(cs, ysrc_row[col], co * (__uint_as_float(r[e]) + g.bias[col]));
-              }
-            }
-          } else {
-            __nv_bfloat16* orow = g.out_bf16 + (size_t)row * g.ld_h;
-            const __nv_bfloat16* rrow = (EPI == EPI_HID) ? g.resid + (size_t)row * g.ld_h : nullptr;
-            const bool vec = (g.ld_h % 8 == 0) && (col0 + 32 <= g.n_out);
-            if (vec) {
-#pragma unroll
-              for (int e = 0; e < 32; e += 8) {
-                float x[8];
-                const float4 b0 = *reinterpret_cast<const float4*>(g.bias + col0 + e);
-                const float4 b1 = *reinterpret_cast<const float4*>(g.bias + col0 + e + 4);
-                const float bb[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
-#pragma unroll
-                for (int u = 0; u < 8; ++u) x[u] = __uint_as_float(r[e + u]) + bb[u];
-                if (EPI == EPI_HID) {
-                  const uint4 rv = *reinterpret_cast<const uint4*>(rrow + col0 + e);
-                  const __nv_bfloat162* rp = reinterpret_cast<const __nv_bfloat162*>(&rv);
-#pragma unroll
-                  for (int u = 0; u < 4; ++u) {
-                    const float2 rf = __bfloat1622float2(rp[u]);
-                    x[2 * u] = rf.x + silu(x[2 * u]);
-                    x[2 * u + 1] = rf.y + silu(x[2 * u + 1]);
-                  }
-                }
-                uint4 ov;
-                __nv_bfloat162* op = reinterpret_cast<__nv_bfloat162*>(&ov);
-#pragma unroll
-                for (int u = 0; u < 4; ++u) op[u] = __floats2bfloat162_rn(x[2 * u], x[2 * u + 1]);
-                *reinterpret_cast<uint4*>(orow + col0 + e) = ov;
-              }
-            } else {
-#pragma unroll
-              for (int e = 0; e < 32; ++e) {
-                const int col = col0 + e;
-                if (col < g.n_out) {
-                  float x = __uint_as_float(r[e]) + g.bias[col];
-                  if (EPI == EPI_HID) x = __bfloat162float(rrow[col]) + silu(x);
-                  orow[col] = __float2bfloat16_rn(x);
-                }
-              }
-            }
-          }
-        }
+        if (row_ok && col0 < g.n_out) epilogue_chunk<EPI>(g, row, col0, r, cs, co, ysrc_row);
       }
       tc_fence_before();
       __syncwarp();
@@ -357,6 +421,176 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)C::kTmemCols)
                  : "memory");
+  }
+}
+
+// ---------------------------------------------------------------------------------------------------
+// CTA-pair kernel for large row counts: a cluster of two CTAs computes a 256 x 256 output tile with
+// tcgen05.mma.cta_group::2.  Each CTA stages only its own 128 rows of A and 128 of the tile's 256
+// weight rows (32 KB per k-block instead of 48 KB for the same 128 x 256 x 64 of tensor work per SM), so
+// the L2 -> shared-memory stream per flop drops by a third.  Rank 0 of the pair issues the MMAs; both
+// CTAs run a TMA warp and four epilogue warps on their own 128 accumulator rows.
+//   full[s]   in rank 0, completed by both CTAs' TMA bytes          empty[s]  in each CTA, MMA commit
+//   accf[b]   in each CTA, MMA commit                               acce[b]   in rank 0, 8 epilogue warps
+// ---------------------------------------------------------------------------------------------------
+constexpr int kPairBN = 256;
+constexpr int kPairStages = 6;
+constexpr int kPairStageBytes = (BM + kPairBN / 2) * BK * 2;
+constexpr int kPairSmemBytes = kPairStages * kPairStageBytes + 1024 + 256;
+
+template <int EPI>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemmThreads, 1)
+gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_w,
+                 const GemmArgs g) {
+  constexpr int BN = kPairBN, S = kPairStages;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t tiles = (raw + 1023u) & ~1023u;
+  uint8_t* aux = smem_raw + (tiles - raw) + S * kPairStageBytes;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(aux);  // full[S], empty[S], acc_full[2], acc_empty[2]
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(aux + 8 * (2 * S + 4));
+  volatile int* dead = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  const uint32_t bar0 = smem_u32(bars);
+  auto full_bar = [&](int s) { return bar0 + 8u * s; };
+  auto empty_bar = [&](int s) { return bar0 + 8u * (S + s); };
+  auto accf_bar = [&](int b) { return bar0 + 8u * (2 * S + b); };
+  auto acce_bar = [&](int b) { return bar0 + 8u * (2 * S + 2 + b); };
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();
+  const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
+  const int m = min(*g.m_dev, g.m_cap);
+  const int tiles_m = (m + 2 * BM - 1) / (2 * BM);
+  const int tiles_n = (g.n_out + BN - 1) / BN;
+  const int n_tiles = tiles_m * tiles_n;
+  const int num_kb = (g.k_dim + BK - 1) / BK;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < S; ++s) {
+      mbar_init(full_bar(s), 1);
+      mbar_init(empty_bar(s), 1);
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(accf_bar(b), 1);
+      mbar_init(acce_bar(b), 8);
+    }
+    *dead = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                 "r"(512u)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  __syncwarp();
+  cluster_sync_all();  // the peer's barriers are initialised before anything arrives on them
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ---------------- TMA producer (both CTAs) ----------------
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      for (int t = pair; t < n_tiles; t += n_pairs) {
+        const int m0 = (t / tiles_n) * (2 * BM) + (int)rank * BM;
+        const int n0 = (t % tiles_n) * BN + (int)rank * (BN / 2);
+        for (int kb = 0; kb < num_kb; ++kb) {
+          mbar_wait(empty_bar(stage), phase ^ 1u, dead, g.err);
+          const uint32_t sa = tiles + stage * kPairStageBytes;
+          const uint32_t sb = sa + BM * BK * 2;
+          const uint32_t full0 = map_to_cta(full_bar(stage), 0);
+          if (rank == 0) mbar_expect_tx(full_bar(stage), 2u * (uint32_t)kPairStageBytes);
+          tma_load_2d_pair(sa, &map_a, full0, kb * BK, m0);
+          tma_load_2d_pair(sb, &map_w, full0, kb * BK, n0);
+          if (++stage == S) {
+            stage = 0;
+            phase ^= 1u;
+          }
+        }
+      }
+      drain_after_timeout(dead);
+    }
+  } else if (warp == 1) {
+    // ---------------- MMA issuer (rank 0 only) ----------------
+    if (rank == 0 && lane == 0) {
+      constexpr uint32_t idesc =
+          (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)((2 * BM) >> 4) << 24);
+      int stage = 0;
+      uint32_t phase = 0;
+      int it = 0;
+      for (int t = pair; t < n_tiles; t += n_pairs, ++it) {
+        const int acc = it & 1;
+        const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
+        mbar_wait(acce_bar(acc), acc_phase ^ 1u, dead, g.err);  // both CTAs' epilogues have drained it
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
+        for (int kb = 0; kb < num_kb; ++kb) {
+          mbar_wait(full_bar(stage), phase, dead, g.err);
+          tc_fence_after();
+          const uint32_t sa = tiles + stage * kPairStageBytes;
+          const uint32_t sb = sa + BM * BK * 2;
+          const uint64_t da = smem_desc_sw128(sa), db = smem_desc_sw128(sb);
+#pragma unroll
+          for (int k = 0; k < BK / UMMA_K; ++k)
+            tc_mma_bf16_pair(d_tmem, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), idesc, (kb | k) != 0 ? 1u : 0u);
+          tc_commit_pair(empty_bar(stage));                 // frees the stage in this CTA ...
+          tc_commit_pair(map_to_cta(empty_bar(stage), 1));  // ... and in the peer
+          if (++stage == S) {
+            stage = 0;
+            phase ^= 1u;
+          }
+        }
+        tc_commit_pair(accf_bar(acc));
+        tc_commit_pair(map_to_cta(accf_bar(acc), 1));
+      }
+    }
+  } else {
+    // ---------------- epilogue warps (both CTAs, own 128 rows) ----------------
+    const int quarter = warp & 3;
+    int it = 0;
+    for (int t = pair; t < n_tiles; t += n_pairs, ++it) {
+      const int m0 = (t / tiles_n) * (2 * BM) + (int)rank * BM, n0 = (t % tiles_n) * BN;
+      const int acc = it & 1;
+      const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
+      mbar_wait(accf_bar(acc), acc_phase, dead, g.err);
+      tc_fence_after();
+      const int row = m0 + quarter * 32 + lane;
+      const bool row_ok = row < m;
+      float cs = 0.f, co = 0.f;
+      const float* ysrc_row = nullptr;
+      if (EPI == EPI_OUT && row_ok) {
+        const int step = g.row_step[row];
+        cs = g.c_skip[step];
+        co = g.c_out[step];
+        ysrc_row = g.ysrc + (size_t)(g.row_map ? g.row_map[row] : row) * g.n_out;
+      }
+#pragma unroll 1
+      for (int c0 = 0; c0 < BN; c0 += 32) {
+        uint32_t r[32];
+        const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN + c0);
+        tc_ld32(taddr, r);
+        tc_wait_ld();
+        const int col0 = n0 + c0;
+        if (row_ok && col0 < g.n_out) epilogue_chunk<EPI>(g, row, col0, r, cs, co, ysrc_row);
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive_cluster(map_to_cta(acce_bar(acc), 0));
+    }
+  }
+
+  // ---------------- tear-down: neither CTA leaves while the pair's MMAs may still touch it ----------------
+  tc_fence_before();
+  __syncthreads();
+  __syncwarp();
+  cluster_sync_all();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
   }
 }
 
@@ -422,8 +656,34 @@ asd_status launch_gemm_t(Ctx* c, const void* a_ptr, int a_cols, const void* w_pt
 }
 
 template <int EPI>
+asd_status launch_gemm_pair(Ctx* c, const void* a_ptr, int a_cols, const void* w_ptr, const GemmArgs& g, int m_bound) {
+  CUtensorMap ma, mw;
+  if (!get_tmap(c, a_ptr, g.m_cap, a_cols, BM, &ma) || !get_tmap(c, w_ptr, g.n_out, a_cols, kPairBN / 2, &mw)) {
+    c->err = "cuTensorMapEncodeTiled failed";
+    return ASD_ERR_CUDA;
+  }
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaFuncSetAttribute(gemm_pair_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, kPairSmemBytes);
+    attr_set = true;
+  }
+  const int tiles = ((m_bound + 2 * BM - 1) / (2 * BM)) * ((g.n_out + kPairBN - 1) / kPairBN);
+  const int pairs = std::max(1, std::min(tiles, c->num_sms / 2));
+  gemm_pair_kernel<EPI><<<2 * pairs, kGemmThreads, kPairSmemBytes, c->stream>>>(ma, mw, g);
+  c->launches++;
+  return ASD_OK;
+}
+
+// The CTA-pair kernel pays off once its 256 x 256 tiles fill the machine at least twice over.
+bool use_pair_kernel(const Ctx* c, int m_bound, int n_out) {
+  const long long tiles = (long long)((m_bound + 2 * BM - 1) / (2 * BM)) * ((n_out + kPairBN - 1) / kPairBN);
+  return n_out % (kPairBN / 2) == 0 && tiles >= 2ll * (c->num_sms / 2);
+}
+
+template <int EPI>
 asd_status launch_gemm(Ctx* c, int bn, const void* a_ptr, int a_cols, const void* w_ptr, const GemmArgs& g,
                        int m_bound) {
+  if (use_pair_kernel(c, m_bound, g.n_out)) return launch_gemm_pair<EPI>(c, a_ptr, a_cols, w_ptr, g, m_bound);
   switch (bn) {
     case 256: return launch_gemm_t<256, EPI>(c, a_ptr, a_cols, w_ptr, g, m_bound);
     case 128: return launch_gemm_t<128, EPI>(c, a_ptr, a_cols, w_ptr, g, m_bound);

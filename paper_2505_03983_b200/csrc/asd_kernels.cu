@@ -1,7 +1,9 @@
 // Elementwise / reduction kernels of the ASD round: bookkeeping (active list, row offsets),
 // draft (Algorithm 1, proposal loop), verify + resample + advance (Algorithms 2 and 3, and the
 // advance step of Algorithm 1), the closed-form posterior means (Eq. 4) and the feature packing
-// of the network denoiser.  fp32 throughout; no fast-math.
+// of the network denoiser.  fp32 throughout; the Gaussian noise uses the special-function unit's
+// approximate lg2 / sqrt / sin / cos (absolute error about 1e-6 per normal), everything that decides an
+// accept test (ln u, the reductions) is plain IEEE fp32.
 #include "asd_internal.h"
 
 namespace asd {
@@ -10,42 +12,66 @@ namespace asd {
 // Counter-based randomness (Algorithm 1, "sample u, xi"): Philox4x32-10, counter =
 // (dimension block, step, chain id, tag).
 // ---------------------------------------------------------------------------------------------
-__device__ __forceinline__ uint4 philox4x32_10(uint4 c, uint32_t k0, uint32_t k1) {
-  constexpr uint32_t M0 = 0xD2511F53u, M1 = 0xCD9E8D57u, W0 = 0x9E3779B9u, W1 = 0xBB67AE85u;
+// Round keys of the ten rounds (key + r * Weyl constant), computed once on the host and passed in
+// the kernel arguments, so a round is two 32x32->64 multiplies and two three-input xors.
+struct PhiloxKeys {
+  uint32_t k[20];
+};
+
+PhiloxKeys make_philox_keys(uint64_t seed) {
+  PhiloxKeys K;
+  uint32_t k0 = (uint32_t)(seed & 0xffffffffull), k1 = (uint32_t)(seed >> 32);
+  for (int r = 0; r < 10; ++r) {
+    K.k[2 * r] = k0;
+    K.k[2 * r + 1] = k1;
+    k0 += 0x9E3779B9u;
+    k1 += 0xBB67AE85u;
+  }
+  return K;
+}
+
+__device__ __forceinline__ uint4 philox4x32_10(uint4 c, const PhiloxKeys& K) {
+  constexpr uint32_t M0 = 0xD2511F53u, M1 = 0xCD9E8D57u;
 #pragma unroll
   for (int r = 0; r < 10; ++r) {
-    const uint32_t hi0 = __umulhi(M0, c.x), lo0 = M0 * c.x;
-    const uint32_t hi1 = __umulhi(M1, c.z), lo1 = M1 * c.z;
-    c = make_uint4(hi1 ^ c.y ^ k0, lo1, hi0 ^ c.w ^ k1, lo0);
-    k0 += W0;
-    k1 += W1;
+    const uint64_t p0 = (uint64_t)M0 * c.x;
+    const uint64_t p1 = (uint64_t)M1 * c.z;
+    c = make_uint4((uint32_t)(p1 >> 32) ^ c.y ^ K.k[2 * r], (uint32_t)p1, (uint32_t)(p0 >> 32) ^ c.w ^ K.k[2 * r + 1],
+                   (uint32_t)p0);
   }
   return c;
 }
 
+// U(r) = ((r >> 9) + 0.5) 2^-23, exactly: the 23 bits become the mantissa of a float in [1, 2) and
+// the subtraction of 1 - 2^-24 is exact (the result has 24 significant bits).
 __device__ __forceinline__ float uniform_from_word(uint32_t r) {
-  return (__uint2float_rn(r >> 9) + 0.5f) * 1.1920928955078125e-07f;  // 2^-23, exact
+  return __uint_as_float((r >> 9) | 0x3f800000u) - 0.99999994f;
 }
 
+// Box-Muller on the special-function unit: radius = sqrt(-2 ln2 lg2 U(r_even)) with lg2.approx and
+// sqrt.approx, angle 2 pi U(r_odd) shifted by -pi into [-pi, pi] (where sin.approx / cos.approx are
+// most accurate); the shift negates both outputs, which the sign of the radius undoes.
 __device__ __forceinline__ void box_muller(uint32_t r_even, uint32_t r_odd, float& n_even, float& n_odd) {
-  const float rad = sqrtf(-2.0f * logf(uniform_from_word(r_even)));
-  float s, c;
-  sincospif(2.0f * uniform_from_word(r_odd), &s, &c);
-  n_even = rad * c;
-  n_odd = rad * s;
+  float rad;
+  asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(rad) : "f"(-1.3862943611198906f * __log2f(uniform_from_word(r_even))));
+  // 2 pi (f - 1 + 2^-24) - pi with f = 1.mantissa in [1, 2)
+  const float th = fmaf(__uint_as_float((r_odd >> 9) | 0x3f800000u), 6.283185307179586f, -9.424777586315302f);
+  n_even = -rad * __cosf(th);
+  n_odd = -rad * __sinf(th);
 }
 
 // xi_step[4q .. 4q+3]
-__device__ __forceinline__ float4 xi4(uint32_t q, uint32_t step, uint32_t chain, uint32_t k0, uint32_t k1) {
-  const uint4 r = philox4x32_10(make_uint4(q, step, chain, 0u), k0, k1);
+__device__ __forceinline__ float4 xi4(uint32_t q, uint32_t step, uint32_t chain, const PhiloxKeys& K) {
+  const uint4 r = philox4x32_10(make_uint4(q, step, chain, 0u), K);
   float4 n;
   box_muller(r.x, r.y, n.x, n.y);
   box_muller(r.z, r.w, n.z, n.w);
   return n;
 }
 
-__device__ __forceinline__ float ln_u(uint32_t step, uint32_t chain, uint32_t k0, uint32_t k1) {
-  const uint4 r = philox4x32_10(make_uint4(0u, step, chain, 1u), k0, k1);
+// ln u_step: evaluated once per slot, with the accurate logarithm (it decides the accept test).
+__device__ __forceinline__ float ln_u(uint32_t step, uint32_t chain, const PhiloxKeys& K) {
+  const uint4 r = philox4x32_10(make_uint4(0u, step, chain, 1u), K);
   return logf(uniform_from_word(r.x));
 }
 
@@ -174,7 +200,7 @@ void launch_prep(Ctx* c, int window) {
 // ---------------------------------------------------------------------------------------------
 struct DraftArgs {
   int d, K, window, nq, vec;
-  uint32_t k0, k1;
+  PhiloxKeys keys;
   uint64_t chain_base;
   const RoundCounters* cnt;
   const int* act;
@@ -208,7 +234,7 @@ __global__ void __launch_bounds__(256) draft_kernel(const DraftArgs A) {
     for (int k = 1; k < w; ++k) {
       const int i = a + k - 1;  // step i -> i+1 uses eta_i, sigma_{i+1}, xi_{i+1}
       const float eta = A.tab.eta[i], sig = A.tab.sig[i];
-      const float4 xi = xi4((uint32_t)q, (uint32_t)(i + 1), chain, A.k0, A.k1);
+      const float4 xi = xi4((uint32_t)q, (uint32_t)(i + 1), chain, A.keys);
       yh.x = fmaf(sig, xi.x, fmaf(eta, v.x, yh.x));
       yh.y = fmaf(sig, xi.y, fmaf(eta, v.y, yh.y));
       yh.z = fmaf(sig, xi.z, fmaf(eta, v.z, yh.z));
@@ -265,8 +291,7 @@ void launch_draft(Ctx* c, int window) {
   A.window = window;
   A.nq = (c->d + 3) / 4;
   A.vec = (c->d % 4 == 0);
-  A.k0 = (uint32_t)(c->seed & 0xffffffffull);
-  A.k1 = (uint32_t)(c->seed >> 32);
+  A.keys = make_philox_keys(c->seed);
   A.chain_base = c->chain_base;
   A.cnt = c->counters;
   A.act = c->act;
@@ -306,7 +331,7 @@ void launch_draft(Ctx* c, int window) {
 // ---------------------------------------------------------------------------------------------
 struct VerifyArgs {
   int d, K, window, nq, vec, use_u;
-  uint32_t k0, k1;
+  PhiloxKeys keys;
   uint64_t chain_base;
   RoundCounters* cnt;
   const int* act;
@@ -341,7 +366,7 @@ __global__ void __launch_bounds__(256) verify_kernel(const VerifyArgs A) {
     // slot 1: proposal mean == target mean, ratio exactly 1 (Lemma 1)
     s_acc[1] = 1;
     A.dbg_lr[(size_t)j * A.window] = 0.f;
-    A.dbg_lu[(size_t)j * A.window] = A.use_u ? ln_u((uint32_t)(a + 1), chain, A.k0, A.k1) : 0.f;
+    A.dbg_lu[(size_t)j * A.window] = A.use_u ? ln_u((uint32_t)(a + 1), chain, A.keys) : 0.f;
   }
   for (int k = 2 + warp; k <= w; k += nwarps) {
     const float* grow = A.G + (size_t)(row0 + k - 2) * A.d;
@@ -349,7 +374,7 @@ __global__ void __launch_bounds__(256) verify_kernel(const VerifyArgs A) {
     for (int q = lane; q < A.nq; q += 32) {
       const float4 v = load4(vrow, q, A.d, A.vec);
       const float4 g = load4(grow, q, A.d, A.vec);
-      const float4 xi = xi4((uint32_t)q, (uint32_t)(a + k), chain, A.k0, A.k1);
+      const float4 xi = xi4((uint32_t)q, (uint32_t)(a + k), chain, A.keys);
       float4 dl = make_float4(v.x - g.x, v.y - g.y, v.z - g.z, v.w - g.w);
       if (!A.vec) {  // ragged tail: dims >= d contribute nothing
         const int b = 4 * q;
@@ -371,7 +396,7 @@ __global__ void __launch_bounds__(256) verify_kernel(const VerifyArgs A) {
     if (lane == 0) {
       const int i = a + k - 1;
       const float lr = -A.tab.c1[i] * dot - A.tab.c2[i] * nrm;
-      const float lu = ln_u((uint32_t)(a + k), chain, A.k0, A.k1);
+      const float lu = ln_u((uint32_t)(a + k), chain, A.keys);
       s_dot[k] = dot;
       s_nrm[k] = nrm;
       s_acc[k] = (lu <= fminf(0.f, lr)) || (nrm == 0.f);
@@ -406,7 +431,7 @@ __global__ void __launch_bounds__(256) verify_kernel(const VerifyArgs A) {
       const float4 b = load4(base, q, A.d, A.vec);
       const float4 g = load4(grow, q, A.d, A.vec);
       const float4 v = load4(vrow, q, A.d, A.vec);
-      const float4 xi = xi4((uint32_t)q, (uint32_t)(i + 1), chain, A.k0, A.k1);
+      const float4 xi = xi4((uint32_t)q, (uint32_t)(i + 1), chain, A.keys);
       float4 o;
       o.x = fmaf(sig, fmaf(-coef, v.x - g.x, xi.x), fmaf(eta, g.x, b.x));
       o.y = fmaf(sig, fmaf(-coef, v.y - g.y, xi.y), fmaf(eta, g.y, b.y));
@@ -422,7 +447,7 @@ __global__ void __launch_bounds__(256) verify_kernel(const VerifyArgs A) {
     for (int q = tid; q < A.nq; q += blockDim.x) {
       const float4 b = load4(base, q, A.d, A.vec);
       const float4 v = load4(vrow, q, A.d, A.vec);
-      const float4 xi = xi4((uint32_t)q, (uint32_t)(i + 1), chain, A.k0, A.k1);
+      const float4 xi = xi4((uint32_t)q, (uint32_t)(i + 1), chain, A.keys);
       float4 o;
       o.x = fmaf(sig, xi.x, fmaf(eta, v.x, b.x));
       o.y = fmaf(sig, xi.y, fmaf(eta, v.y, b.y));
@@ -450,8 +475,7 @@ void launch_verify(Ctx* c, int window, bool use_u) {
   A.nq = (c->d + 3) / 4;
   A.vec = (c->d % 4 == 0);
   A.use_u = use_u;
-  A.k0 = (uint32_t)(c->seed & 0xffffffffull);
-  A.k1 = (uint32_t)(c->seed >> 32);
+  A.keys = make_philox_keys(c->seed);
   A.chain_base = c->chain_base;
   A.cnt = c->counters;
   A.act = c->act;

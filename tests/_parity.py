@@ -20,11 +20,48 @@ def tolerances(kind: str):
     return 1e-4, 1e-4
 
 
+EPS_BF16 = 2.0 ** -8
+
+
+def ln_ratio_tolerance(wl, sch, rec, cascade=False):
+    """Per-slot tolerance on ln ratio: 1e-4 max(1, |ln ratio|) for the fp32 drifts, 2e-3 max(1, |ln ratio|)
+    for the bf16 network.
+
+    cascade=True (the 6-layer, width-4096 network only) widens it: two implementations that accumulate in a
+    different order round a few hidden units to different bf16 values; the next layer's
+    pre-activations all move a little, which flips more roundings, and after a few layers the
+    hidden states differ like independent bf16 roundings: the network branch n = g - c_skip y of the
+    drift is reproducible only to about 2^-8 |n| (observed 0.7 * 2^-8 between fp32 and fp64
+    accumulation on the CPU at width 4096, 6 layers).  With delta = v_a - g_{k-1} perturbed by an
+    isotropic e_k = 2^-8 (|n_a| + |n_{k-1}|), ln ratio = -(eta/sigma) <xi, delta> - (eta/sigma)^2 |delta|^2 / 2
+    moves by at most (5 sigma of the two inner products)
+        (eta/sigma) 5 e_k + (eta/sigma)^2 (5 |delta| e_k / sqrt(d) + e_k^2 / 2).
+    The tolerance is then the larger of that and 2e-3 max(1, |ln ratio|)."""
+    w = rec.w
+    if wl.kind != "mlp":
+        return 1e-4 * np.maximum(1.0, np.abs(rec.ln_ratio))
+    tol = 2e-3 * np.maximum(1.0, np.abs(rec.ln_ratio))
+    if not cascade:
+        return tol
+    c_skip = np.asarray(wl.c_skip, dtype=np.float64)
+    a = rec.a_before
+    n0 = np.linalg.norm(rec.drift[0] - c_skip[a] * rec.points[0])
+    for k in range(1, w):
+        i = a + k
+        nk = np.linalg.norm(rec.drift[k] - c_skip[i] * rec.points[k])
+        delta = np.linalg.norm(rec.drift[0] - rec.drift[k])
+        e = EPS_BF16 * (n0 + nk)
+        r = sch.eta[i] / sch.sigma[i]
+        tol[k] = max(tol[k], r * 5 * e + r * r * (5 * delta * e / math.sqrt(wl.d) + 0.5 * e * e))
+    return tol
+
+
 def rel_l2(a, b):
     return float(np.linalg.norm(a - b) / max(np.linalg.norm(b), 1e-6))
 
 
-def lockstep(sampler, wl, n_chains, n_rounds, chain_base=0, check_chains=None, cond=None, log=None):
+def lockstep(sampler, wl, n_chains, n_rounds, chain_base=0, check_chains=None, cond=None, log=None,
+             cascade=False):
     """Runs `n_rounds` rounds on the GPU; before each round the oracle is restarted from the
     GPU's state and must reproduce ln u, ln ratio, the accepted prefix and the new state."""
     g = oden.from_workload(wl)
@@ -32,7 +69,7 @@ def lockstep(sampler, wl, n_chains, n_rounds, chain_base=0, check_chains=None, c
     tol_y, tol_r = tolerances(wl.kind)
     check = list(range(n_chains)) if check_chains is None else list(check_chains)
     sampler.reset(n_chains, chain_base, cond=cond)
-    worst = dict(y=0.0, lr=0.0, lu=0.0, exempt=0, decided=0, rounds=0)
+    worst = dict(y=0.0, lr=0.0, lr_over_tol=0.0, lu=0.0, exempt=0, decided=0, rounds=0)
     for r in range(n_rounds):
         a0, y0, _ = [t.cpu().numpy() for t in sampler.get_state()]
         st = sampler.round()
@@ -53,12 +90,19 @@ def lockstep(sampler, wl, n_chains, n_rounds, chain_base=0, check_chains=None, c
                                  sampler.window)
             w = rec.w
             e_lu = np.max(np.abs(lu[j, :w] - rec.ln_u) / np.maximum(1.0, np.abs(rec.ln_u)))
-            e_lr = np.max(np.abs(lr[j, :w] - rec.ln_ratio) / np.maximum(1.0, np.abs(rec.ln_ratio)))
+            d_lr = np.abs(lr[j, :w] - rec.ln_ratio)
+            tol_lr = ln_ratio_tolerance(wl, sch, rec, cascade)
+            e_lr = np.max(d_lr / np.maximum(1.0, np.abs(rec.ln_ratio)))
             worst["lu"] = max(worst["lu"], e_lu)
             worst["lr"] = max(worst["lr"], e_lr)
+            worst["lr_over_tol"] = max(worst["lr_over_tol"], float(np.max(d_lr / tol_lr)))
             assert e_lu < 1e-5, (r, j, e_lu)
-            assert e_lr < tol_r, (r, j, e_lr, lr[j, :w], rec.ln_ratio)
-            if rec.margin > MARGIN:
+            assert np.all(d_lr < tol_lr), (r, j, d_lr / tol_lr, lr[j, :w], rec.ln_ratio)
+            # a decision is compared bit-exactly unless it lies within the margin: 1e-3, or with
+            # cascade=True the reproducibility bound of ln ratio where that is larger
+            last = min(rec.n + 1, w)
+            slack = np.abs(rec.ln_ratio[1:last] - rec.ln_u[1:last]) - np.maximum(MARGIN, tol_lr[1:last] if cascade else 0.0)
+            if last < 2 or np.all(slack > 0):
                 worst["decided"] += 1
                 assert acc[j] == rec.n, (r, j, acc[j], rec.n, rec.margin)
             else:
