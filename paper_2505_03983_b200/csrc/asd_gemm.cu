@@ -204,7 +204,9 @@ struct Cfg {
   static constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
 };
 
-__device__ __forceinline__ float silu(float z) { return z / (1.0f + __expf(-z)); }
+// SiLU on the un-rounded fp32 accumulator; ex2.approx and rcp.approx (relative error ~2^-22, far below
+// the bf16 rounding that follows).
+__device__ __forceinline__ float silu(float z) { return __fdividef(z, 1.0f + __expf(-z)); }
 
 // Epilogue of 32 consecutive accumulator columns [col0, col0 + 32) of one output row held by this
 // thread: bias, then the layer's fused tail, then the store (16-byte vectors where the shape allows).
@@ -273,6 +275,104 @@ __device__ __forceinline__ void epilogue_chunk(const GemmArgs& g, int row, int c
           orow[col] = __float2bfloat16_rn(x);
         }
       }
+    }
+  }
+}
+
+// What the fused tail of a layer reads from global memory for 32 columns of one row: the residual
+// h_{l-1} (32 bf16) for EPI_HID, the state y (32 fp32) for EPI_OUT, nothing for EPI_IN.  Fetched one
+// chunk ahead of the arithmetic so that its latency overlaps the previous chunk.
+template <int EPI>
+struct EpiOperand {
+  uint4 v[EPI == EPI_OUT ? 8 : (EPI == EPI_HID ? 4 : 1)];
+};
+
+template <int EPI>
+__device__ __forceinline__ void epi_fetch(EpiOperand<EPI>& op, const GemmArgs& g, int row, int col0, const float* ysrc_row) {
+  if (EPI == EPI_HID) {
+    const uint4* p = reinterpret_cast<const uint4*>(g.resid + (size_t)row * g.ld_h + col0);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) op.v[i] = p[i];
+  } else if (EPI == EPI_OUT) {
+    const uint4* p = reinterpret_cast<const uint4*>(ysrc_row + col0);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) op.v[i] = p[i];
+  }
+}
+
+// The 16-byte-vector epilogue of 32 full columns with the operand already in registers.
+template <int EPI>
+__device__ __forceinline__ void epi_apply(const GemmArgs& g, int row, int col0, const uint32_t (&r)[32],
+                                          const EpiOperand<EPI>& op, float cs, float co) {
+  if (EPI == EPI_OUT) {
+    float* orow = g.out_f32 + (size_t)row * g.n_out + col0;
+#pragma unroll
+    for (int e = 0; e < 32; e += 4) {
+      const float4 b4 = *reinterpret_cast<const float4*>(g.bias + col0 + e);
+      const uint4 yv = op.v[e >> 2];
+      float4 o;
+      o.x = fmaf(cs, __uint_as_float(yv.x), co * (__uint_as_float(r[e + 0]) + b4.x));
+      o.y = fmaf(cs, __uint_as_float(yv.y), co * (__uint_as_float(r[e + 1]) + b4.y));
+      o.z = fmaf(cs, __uint_as_float(yv.z), co * (__uint_as_float(r[e + 2]) + b4.z));
+      o.w = fmaf(cs, __uint_as_float(yv.w), co * (__uint_as_float(r[e + 3]) + b4.w));
+      *reinterpret_cast<float4*>(orow + e) = o;
+    }
+  } else {
+    __nv_bfloat16* orow = g.out_bf16 + (size_t)row * g.ld_h + col0;
+#pragma unroll
+    for (int e = 0; e < 32; e += 8) {
+      float x[8];
+      const float4 b0 = *reinterpret_cast<const float4*>(g.bias + col0 + e);
+      const float4 b1 = *reinterpret_cast<const float4*>(g.bias + col0 + e + 4);
+      const float bb[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
+#pragma unroll
+      for (int u = 0; u < 8; ++u) x[u] = __uint_as_float(r[e + u]) + bb[u];
+      if (EPI == EPI_HID) {
+        const uint4 rv = op.v[e >> 3];
+        const __nv_bfloat162* rp = reinterpret_cast<const __nv_bfloat162*>(&rv);
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const float2 rf = __bfloat1622float2(rp[u]);
+          x[2 * u] = rf.x + silu(x[2 * u]);
+          x[2 * u + 1] = rf.y + silu(x[2 * u + 1]);
+        }
+      }
+      uint4 ov;
+      __nv_bfloat162* op2 = reinterpret_cast<__nv_bfloat162*>(&ov);
+#pragma unroll
+      for (int u = 0; u < 4; ++u) op2[u] = __floats2bfloat162_rn(x[2 * u], x[2 * u + 1]);
+      *reinterpret_cast<uint4*>(orow + e) = ov;
+    }
+  }
+}
+
+// Epilogue of one accumulator tile row: this thread owns output row `row` (tensor-memory lane) and walks
+// its BN columns in chunks of 32.  tcgen05.ld is warp-collective, so every lane runs the loop and only
+// the global accesses are predicated on row_ok.
+template <int EPI, int BN>
+__device__ __forceinline__ void epilogue_tile(const GemmArgs& g, uint32_t taddr0, int row, bool row_ok, int n0, float cs,
+                                              float co, const float* ysrc_row) {
+  const bool full_vec =
+      (n0 + BN <= g.n_out) && (EPI == EPI_OUT ? (g.n_out % 4 == 0) : (g.ld_h % 8 == 0));  // warp-uniform
+  if (full_vec) {
+    EpiOperand<EPI> op[2];
+    if (row_ok) epi_fetch<EPI>(op[0], g, row, n0, ysrc_row);
+#pragma unroll
+    for (int c = 0; c < BN / 32; ++c) {
+      uint32_t r[32];
+      tc_ld32(taddr0 + (uint32_t)(c * 32), r);
+      if (c + 1 < BN / 32 && row_ok) epi_fetch<EPI>(op[(c + 1) & 1], g, row, n0 + (c + 1) * 32, ysrc_row);
+      tc_wait_ld();
+      if (row_ok) epi_apply<EPI>(g, row, n0 + c * 32, r, op[c & 1], cs, co);
+    }
+  } else {
+#pragma unroll 1
+    for (int c0 = 0; c0 < BN; c0 += 32) {
+      uint32_t r[32];
+      tc_ld32(taddr0 + (uint32_t)c0, r);
+      tc_wait_ld();
+      const int col0 = n0 + c0;
+      if (row_ok && col0 < g.n_out) epilogue_chunk<EPI>(g, row, col0, r, cs, co, ysrc_row);
     }
   }
 }
@@ -399,15 +499,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         co = g.c_out[step];
         ysrc_row = g.ysrc + (size_t)(g.row_map ? g.row_map[row] : row) * g.n_out;
       }
-#pragma unroll 1
-      for (int c0 = 0; c0 < BN; c0 += 32) {
-        uint32_t r[32];
-        const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN + c0);
-        tc_ld32(taddr, r);
-        tc_wait_ld();
-        const int col0 = n0 + c0;
-        if (row_ok && col0 < g.n_out) epilogue_chunk<EPI>(g, row, col0, r, cs, co, ysrc_row);
-      }
+      epilogue_tile<EPI, BN>(g, tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN), row, row_ok, n0, cs,
+                             co, ysrc_row);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(acce_bar(acc));
@@ -568,15 +661,8 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
         co = g.c_out[step];
         ysrc_row = g.ysrc + (size_t)(g.row_map ? g.row_map[row] : row) * g.n_out;
       }
-#pragma unroll 1
-      for (int c0 = 0; c0 < BN; c0 += 32) {
-        uint32_t r[32];
-        const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN + c0);
-        tc_ld32(taddr, r);
-        tc_wait_ld();
-        const int col0 = n0 + c0;
-        if (row_ok && col0 < g.n_out) epilogue_chunk<EPI>(g, row, col0, r, cs, co, ysrc_row);
-      }
+      epilogue_tile<EPI, BN>(g, tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN), row, row_ok, n0, cs,
+                             co, ysrc_row);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive_cluster(map_to_cta(acce_bar(acc), 0));
