@@ -15,6 +15,9 @@
 // ASD_ERR_TIMEOUT in the context's device error word and carries on as if the wait had
 // completed, so the kernel always reaches its tear-down (tensor memory is released) and the host
 // reports the error after the call.
+#include <stdlib.h>
+#include <string.h>
+
 #include <algorithm>
 
 #include "asd_internal.h"
@@ -518,28 +521,32 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
 }
 
 // ---------------------------------------------------------------------------------------------------
-// CTA-pair kernel for large row counts: a cluster of two CTAs computes a 256 x 256 output tile with
-// tcgen05.mma.cta_group::2.  Each CTA stages only its own 128 rows of A and 128 of the tile's 256
-// weight rows (32 KB per k-block instead of 48 KB for the same 128 x 256 x 64 of tensor work per SM), so
-// the L2 -> shared-memory stream per flop drops by a third.  Rank 0 of the pair issues the MMAs; both
+// CTA-pair kernel: a cluster of two CTAs computes a 256 x BN output tile with tcgen05.mma.cta_group::2.
+// Each CTA stages only its own 128 rows of A and BN/2 of the tile's BN weight rows (for BN = 256: 32 KB
+// per k-block instead of 48 KB for the same 128 x 256 x 64 of tensor work per SM), so the L2 -> shared-memory
+// stream per flop drops by a third.  Rank 0 of the pair issues the MMAs; both
 // CTAs run a TMA warp and four epilogue warps on their own 128 accumulator rows.
 //   full[s]   in rank 0, completed by both CTAs' TMA bytes          empty[s]  in each CTA, MMA commit
 //   accf[b]   in each CTA, MMA commit                               acce[b]   in rank 0, 8 epilogue warps
 // ---------------------------------------------------------------------------------------------------
-constexpr int kPairBN = 256;
-constexpr int kPairStages = 6;
-constexpr int kPairStageBytes = (BM + kPairBN / 2) * BK * 2;
-constexpr int kPairSmemBytes = kPairStages * kPairStageBytes + 1024 + 256;
+template <int BN>
+struct PairCfg {
+  static constexpr int kStageBytes = (BM + BN / 2) * BK * 2;           // per CTA: 128 rows of A, BN/2 rows of W
+  static constexpr int kStages = (BN >= 256) ? 6 : (BN >= 128) ? 8 : 9;  // <= 192 KB of stages
+  static constexpr int kTmemCols = 2 * BN;                             // two accumulators per CTA
+  static constexpr int kSmemBytes = kStages * kStageBytes + 1024 + 256;
+};
 
-template <int EPI>
+template <int BN, int EPI>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemmThreads, 1)
 gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_w,
                  const GemmArgs g) {
-  constexpr int BN = kPairBN, S = kPairStages;
+  using C = PairCfg<BN>;
+  constexpr int S = C::kStages;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t tiles = (raw + 1023u) & ~1023u;
-  uint8_t* aux = smem_raw + (tiles - raw) + S * kPairStageBytes;
+  uint8_t* aux = smem_raw + (tiles - raw) + S * C::kStageBytes;
   uint64_t* bars = reinterpret_cast<uint64_t*>(aux);  // full[S], empty[S], acc_full[2], acc_empty[2]
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(aux + 8 * (2 * S + 4));
   volatile int* dead = reinterpret_cast<volatile int*>(tmem_slot + 1);
@@ -572,7 +579,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
   }
   if (warp == 1) {
     asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
-                 "r"(512u)
+                 "r"((uint32_t)C::kTmemCols)
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
   }
@@ -593,10 +600,10 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
         const int n0 = (t % tiles_n) * BN + (int)rank * (BN / 2);
         for (int kb = 0; kb < num_kb; ++kb) {
           mbar_wait(empty_bar(stage), phase ^ 1u, dead, g.err);
-          const uint32_t sa = tiles + stage * kPairStageBytes;
+          const uint32_t sa = tiles + stage * C::kStageBytes;
           const uint32_t sb = sa + BM * BK * 2;
           const uint32_t full0 = map_to_cta(full_bar(stage), 0);
-          if (rank == 0) mbar_expect_tx(full_bar(stage), 2u * (uint32_t)kPairStageBytes);
+          if (rank == 0) mbar_expect_tx(full_bar(stage), 2u * (uint32_t)C::kStageBytes);
           tma_load_2d_pair(sa, &map_a, full0, kb * BK, m0);
           tma_load_2d_pair(sb, &map_w, full0, kb * BK, n0);
           if (++stage == S) {
@@ -624,7 +631,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
         for (int kb = 0; kb < num_kb; ++kb) {
           mbar_wait(full_bar(stage), phase, dead, g.err);
           tc_fence_after();
-          const uint32_t sa = tiles + stage * kPairStageBytes;
+          const uint32_t sa = tiles + stage * C::kStageBytes;
           const uint32_t sb = sa + BM * BK * 2;
           const uint64_t da = smem_desc_sw128(sa), db = smem_desc_sw128(sb);
 #pragma unroll
@@ -676,7 +683,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
   cluster_sync_all();
   if (warp == 1) {
     tc_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)C::kTmemCols) : "memory");
   }
 }
 
@@ -741,52 +748,80 @@ asd_status launch_gemm_t(Ctx* c, const void* a_ptr, int a_cols, const void* w_pt
   return ASD_OK;
 }
 
-template <int EPI>
-asd_status launch_gemm_pair(Ctx* c, const void* a_ptr, int a_cols, const void* w_ptr, const GemmArgs& g, int m_bound) {
+template <int BN, int EPI>
+asd_status launch_gemm_pair_t(Ctx* c, const void* a_ptr, int a_cols, const void* w_ptr, const GemmArgs& g, int m_bound) {
+  using C = PairCfg<BN>;
   CUtensorMap ma, mw;
-  if (!get_tmap(c, a_ptr, g.m_cap, a_cols, BM, &ma) || !get_tmap(c, w_ptr, g.n_out, a_cols, kPairBN / 2, &mw)) {
+  if (!get_tmap(c, a_ptr, g.m_cap, a_cols, BM, &ma) || !get_tmap(c, w_ptr, g.n_out, a_cols, BN / 2, &mw)) {
     c->err = "cuTensorMapEncodeTiled failed";
     return ASD_ERR_CUDA;
   }
   static bool attr_set = false;
   if (!attr_set) {
-    cudaFuncSetAttribute(gemm_pair_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, kPairSmemBytes);
+    cudaFuncSetAttribute(gemm_pair_kernel<BN, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
     attr_set = true;
   }
-  const int tiles = ((m_bound + 2 * BM - 1) / (2 * BM)) * ((g.n_out + kPairBN - 1) / kPairBN);
+  const int tiles = ((m_bound + 2 * BM - 1) / (2 * BM)) * ((g.n_out + BN - 1) / BN);
   const int pairs = std::max(1, std::min(tiles, c->num_sms / 2));
-  gemm_pair_kernel<EPI><<<2 * pairs, kGemmThreads, kPairSmemBytes, c->stream>>>(ma, mw, g);
+  gemm_pair_kernel<BN, EPI><<<2 * pairs, kGemmThreads, C::kSmemBytes, c->stream>>>(ma, mw, g);
   c->launches++;
   return ASD_OK;
 }
 
-// The CTA-pair kernel pays off once its 256 x 256 tiles fill the machine at least twice over.
-bool use_pair_kernel(const Ctx* c, int m_bound, int n_out) {
-  const long long tiles = (long long)((m_bound + 2 * BM - 1) / (2 * BM)) * ((n_out + kPairBN - 1) / kPairBN);
-  return n_out % (kPairBN / 2) == 0 && tiles >= 2ll * (c->num_sms / 2);
+// Which kernel and column-tile width serve a [m x k] x [n x k]^T product best.  Model: every SM fills
+// its shared memory from L2 at about 50 bytes per clock and its tensor pipe retires a 128 x 256 x 64
+// block in 512 clocks; a launch takes (waves of tiles) x (k-blocks) x max(fill, math) clocks.
+struct GemmPlan {
+  bool pair;
+  int bn;
+};
+
+GemmPlan plan_gemm(const Ctx* c, int m_bound, int n_out) {
+  static const int mode = [] {
+    const char* e = getenv("ASD_GEMM_MODE");  // tuning aid: "cta" or "pair" pins the kernel family
+    return !e ? 0 : (!strcmp(e, "cta") ? 1 : (!strcmp(e, "pair") ? 2 : 0));
+  }();
+  const double fill_rate = 50.0;
+  GemmPlan best{false, 32};
+  double best_t = 1e300;
+  const int cand[4] = {256, 128, 64, 32};
+  for (int pair = 0; pair < 2; ++pair) {
+    if ((mode == 1 && pair) || (mode == 2 && !pair)) continue;
+    const int units = pair ? c->num_sms / 2 : c->num_sms;
+    const int tm = pair ? 2 * BM : BM;
+    for (int i = 0; i < (pair ? 3 : 4); ++i) {
+      const int bn = cand[i];
+      if (pair && n_out % (bn / 2) != 0) continue;  // each CTA of a pair stages a whole half tile of W
+      const long long tiles = (long long)((m_bound + tm - 1) / tm) * ((n_out + bn - 1) / bn);
+      const double waves = (double)((tiles + units - 1) / units);
+      const double fill = (BM + (pair ? bn / 2 : bn)) * (BK * 2) / fill_rate;
+      const double math = 512.0 * bn / 256.0;
+      const double t = waves * std::max(fill, math);
+      if (t < best_t * 0.999) {
+        best_t = t;
+        best = GemmPlan{pair != 0, bn};
+      }
+    }
+  }
+  return best;
 }
 
 template <int EPI>
-asd_status launch_gemm(Ctx* c, int bn, const void* a_ptr, int a_cols, const void* w_ptr, const GemmArgs& g,
-                       int m_bound) {
-  if (use_pair_kernel(c, m_bound, g.n_out)) return launch_gemm_pair<EPI>(c, a_ptr, a_cols, w_ptr, g, m_bound);
-  switch (bn) {
+asd_status launch_gemm(Ctx* c, const void* a_ptr, int a_cols, const void* w_ptr, const GemmArgs& g, int m_bound) {
+  const GemmPlan p = plan_gemm(c, m_bound, g.n_out);
+  if (p.pair) {
+    switch (p.bn) {
+      case 256: return launch_gemm_pair_t<256, EPI>(c, a_ptr, a_cols, w_ptr, g, m_bound);
+      case 128: return launch_gemm_pair_t<128, EPI>(c, a_ptr, a_cols, w_ptr, g, m_bound);
+      default: return launch_gemm_pair_t<64, EPI>(c, a_ptr, a_cols, w_ptr, g, m_bound);
+    }
+  }
+  switch (p.bn) {
     case 256: return launch_gemm_t<256, EPI>(c, a_ptr, a_cols, w_ptr, g, m_bound);
     case 128: return launch_gemm_t<128, EPI>(c, a_ptr, a_cols, w_ptr, g, m_bound);
     case 64: return launch_gemm_t<64, EPI>(c, a_ptr, a_cols, w_ptr, g, m_bound);
     default: return launch_gemm_t<32, EPI>(c, a_ptr, a_cols, w_ptr, g, m_bound);
   }
-}
-
-// Column-tile width: the widest tile that still gives every SM a tile.
-int pick_bn(const Ctx* c, int m_bound, int n_out) {
-  const int tiles_m = (m_bound + BM - 1) / BM;
-  const int cand[4] = {256, 128, 64, 32};
-  for (int i = 0; i < 4; ++i) {
-    const int bn = cand[i];
-    if (tiles_m * ((n_out + bn - 1) / bn) >= c->num_sms) return bn;
-  }
-  return 32;
 }
 
 }  // namespace
@@ -806,12 +841,11 @@ asd_status mlp_forward(Ctx* c, const RowSet& rs, float* out, int pass) {
   g.bias = M.b_in;
   g.out_bf16 = M.H[0];
   g.ld_h = M.width;
-  const int bn_h = pick_bn(c, m_bound, M.width);
   const int ph_in = pass == 0 ? PH_D1_IN : PH_D2_IN, ph_hid = pass == 0 ? PH_D1_HID : PH_D2_HID,
             ph_out = pass == 0 ? PH_D1_OUT : PH_D2_OUT;
   {
     ProfScope ps(pass < 2 ? c : nullptr, ph_in);
-    st = launch_gemm<EPI_IN>(c, bn_h, M.X, M.in_pad, M.W_in, g, m_bound);
+    st = launch_gemm<EPI_IN>(c, M.X, M.in_pad, M.W_in, g, m_bound);
   }
   if (st != ASD_OK) return st;
   ProfScope ps_hid(pass < 2 ? c : nullptr, ph_hid);
@@ -821,7 +855,7 @@ asd_status mlp_forward(Ctx* c, const RowSet& rs, float* out, int pass) {
     g.bias = M.b_hid + (size_t)l * M.width;
     g.resid = M.H[l & 1];
     g.out_bf16 = M.H[(l + 1) & 1];
-    st = launch_gemm<EPI_HID>(c, bn_h, M.H[l & 1], M.width, M.W_hid + (size_t)l * M.width * M.width, g, m_bound);
+    st = launch_gemm<EPI_HID>(c, M.H[l & 1], M.width, M.W_hid + (size_t)l * M.width * M.width, g, m_bound);
     if (st != ASD_OK) return st;
   }
   ps_hid.~ProfScope();
@@ -838,9 +872,8 @@ asd_status mlp_forward(Ctx* c, const RowSet& rs, float* out, int pass) {
   g.row_step = rs.row_step;
   g.c_skip = c->tab.c_skip;
   g.c_out = c->tab.c_out;
-  const int bn_o = pick_bn(c, m_bound, c->d);
   ProfScope ps_out(pass < 2 ? c : nullptr, ph_out);
-  return launch_gemm<EPI_OUT>(c, bn_o, M.H[M.n_layers & 1], M.width, M.W_out, g, m_bound);
+  return launch_gemm<EPI_OUT>(c, M.H[M.n_layers & 1], M.width, M.W_out, g, m_bound);
 }
 
 }  // namespace asd
