@@ -175,12 +175,13 @@ def run_ours(args):
     barrier()
     clocks.start()
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    launches, rounds_mean, rounds_max, rows = 0, [], [], 0
+    launches, rounds_mean, rounds_max, rows, rows_ver = 0, [], [], 0, 0
     ev0.record()
     for _ in range(args.steps):
         y, r, st = step()
         launches += st.launches
         rounds_mean.append(st.rounds_mean); rounds_max.append(st.rounds_max); rows += st.rows_total
+        rows_ver += st.rows_verified
     ev1.record()
     barrier()
     clk = clocks.stop()
@@ -228,6 +229,7 @@ def run_ours(args):
         "rounds_per_sample": float(np.mean(rounds_mean)), "rounds_max": int(max(rounds_max)),
         "K_over_rounds": wl.K / float(np.mean(rounds_mean)),
         "drift_rows_per_sample_over_K": rows / (args.steps * n * wl.K),
+        "verified_rows_over_drafted_rows": rows_ver / max(rows - args.steps * n * float(np.mean(rounds_mean)), 1.0),
         "gpu_launches": int(launches),
         "clocks": clk,
         "e2e": {"value": total / (ms_e2e / 1e3), "unit": UNIT,
@@ -250,9 +252,10 @@ def run_ours(args):
                             "launches": hid["launches"], "avg_launch_ms": hid["ms"] / max(hid["launches"], 1),
                             "traffic": None}
         ver = prof["verify"]
-        # algorithmic bytes of verify: read G once (4 d (w-1) per chain-round = 4 d per pass-2 row),
-        # read y and v, write y (3 * 4 d per chain-round)
-        vbytes = 4.0 * wl.d * (prof["pass2_gemm_out"]["rows"] + 3 * ver["rows"])
+        # bytes the verify kernel has to move: every drift row it reads (it stops after the first
+        # rejection, so this is less than the 4 d (w - 1) per chain-round of reading the whole window),
+        # plus y^/v reads and the y write (3 * 4 d per chain-round)
+        vbytes = 4.0 * wl.d * (rows_ver + 3 * ver["rows"])
         vach = vbytes / (ver["ms"] / 1e3) / 1e9 if ver["ms"] > 0 else 0.0
         line["roofline_verify"] = {"kernel": "verify_kernel", "bound": "hbm", "achieved": vach, "peak": peaks["hbm_gbs"],
                                    "unit": "GB/s", "frac": vach / peaks["hbm_gbs"], "peak_source": peaks["source"],
@@ -260,8 +263,7 @@ def run_ours(args):
                                    "traffic": None}
     else:
         ver = prof["verify"]
-        rows2 = prof["pass2_closed_form"]["rows"]
-        vbytes = 4.0 * wl.d * (rows2 + 3 * ver["rows"])
+        vbytes = 4.0 * wl.d * (rows_ver + 3 * ver["rows"])
         vach = vbytes / (ver["ms"] / 1e3) / 1e9 if ver["ms"] > 0 else 0.0
         line["roofline"] = {"kernel": "verify_kernel", "bound": "hbm", "achieved": vach, "peak": peaks["hbm_gbs"],
                             "unit": "GB/s", "frac": vach / peaks["hbm_gbs"], "peak_source": peaks["source"],

@@ -110,8 +110,17 @@ typedef struct {
                            (stochastic localization: increments have variance eta, Theorem 2) */
   uint64_t seed;        /* Philox key */
   asd_denoiser den;
-  uint32_t flags;       /* reserved, pass 0 */
+  uint32_t flags;       /* 0 or ASD_FLAG_* */
 } asd_config;
+
+/*
+ * ASD_FLAG_DEBUG_ALL_SLOTS: the Verifier (Algorithm 2) only needs the end of the all-accepted prefix,
+ * so by default the verify kernel stops at the first rejected slot and never reads the drifts
+ * beyond it.  With this flag every slot of the window goes through the accept test of Algorithm 3
+ * (as Algorithm 2 is written) so that asd_debug_last_round returns ln ratio for all of them.  The
+ * chain states are identical either way.
+ */
+#define ASD_FLAG_DEBUG_ALL_SLOTS 1u
 
 typedef struct {
   int32_t n_active_before; /* chains with a < K when the round started */
@@ -127,6 +136,7 @@ typedef struct {
   int64_t rows_total;   /* drift evaluations made, both passes */
   double ms_total;      /* device time of the call, CUDA events on the context's stream */
   int64_t launches;     /* kernels launched by the call */
+  int64_t rows_verified; /* drafted-point drifts the Verifier read (it stops after the first rejection) */
 } asd_run_stats;
 
 /* Library version string (static storage). */
@@ -193,8 +203,9 @@ asd_status asd_set_state(asd_ctx* ctx, const int32_t* a_dev, const float* y_dev,
 /*
  * Diagnostics of the last round, indexed by chain position: ln ratio (Algorithm 3) and
  * ln u per window slot ([n*window] fp32 each; slots beyond the chain's window are not
- * written) and the accepted prefix length n ([n] int32; -1 for chains that were inactive).
- * Device buffers, any may be NULL.
+ * written; ln ratio of slots after the first rejected one is NaN unless the context was
+ * created with ASD_FLAG_DEBUG_ALL_SLOTS) and the accepted prefix length n ([n] int32; -1 for
+ * chains that were inactive).  Device buffers, any may be NULL.
  */
 asd_status asd_debug_last_round(asd_ctx* ctx, float* ln_ratio_dev, float* ln_u_dev, int32_t* accepted_dev);
 

@@ -23,6 +23,7 @@ EXPORTED_SYMBOLS = [
 STATUS = {0: "ASD_OK", 1: "ASD_ERR_INVALID_ARG", 2: "ASD_ERR_UNSUPPORTED", 3: "ASD_ERR_OOM",
           4: "ASD_ERR_CUDA", 5: "ASD_ERR_STATE", 6: "ASD_ERR_TIMEOUT"}
 KIND = {"gmm": 0, "gauss": 1, "mlp": 2}
+FLAG_DEBUG_ALL_SLOTS = 1   # ASD_FLAG_DEBUG_ALL_SLOTS
 
 
 class AsdError(RuntimeError):
@@ -57,7 +58,7 @@ class _RoundStats(C.Structure):
 
 class _RunStats(C.Structure):
     _fields_ = [("rounds_max", C.c_int64), ("rounds_mean", C.c_double), ("rows_total", C.c_int64),
-                ("ms_total", C.c_double), ("launches", C.c_int64)]
+                ("ms_total", C.c_double), ("launches", C.c_int64), ("rows_verified", C.c_int64)]
 
 
 class _PhaseTime(C.Structure):
@@ -80,6 +81,7 @@ class RunStats:
     rows_total: int
     ms_total: float
     launches: int
+    rows_verified: int = 0
 
 
 def lib_path() -> str:
@@ -145,7 +147,7 @@ class AsdSampler:
     denoiser arrays).  Methods mirror the C entry points; tensors are torch CUDA tensors."""
 
     def __init__(self, wl, max_chains: Optional[int] = None, window: Optional[int] = None,
-                 seed: Optional[int] = None, sigma2: Optional[np.ndarray] = None, stream=None):
+                 seed: Optional[int] = None, sigma2: Optional[np.ndarray] = None, stream=None, flags: int = 0):
         import torch
         if not torch.cuda.is_available():
             raise AsdError(4, "no CUDA device: the ASD library has no CPU path")
@@ -187,7 +189,7 @@ class AsdSampler:
         cfg.sigma2 = None if sigma2 is None else f64(sigma2)
         cfg.seed = int(seed if seed is not None else wl.seed)
         cfg.den = den
-        cfg.flags = 0
+        cfg.flags = int(flags)
         self.seed = cfg.seed
         self.stream = stream
         sptr = C.c_void_p(stream.cuda_stream) if stream is not None else C.c_void_p(
@@ -244,7 +246,7 @@ class AsdSampler:
         return RoundStats(rs.n_active_before, rs.n_active_after, rs.rows_pass1, rs.rows_pass2, rs.accepted_total)
 
     def _run_stats(self, s: _RunStats) -> RunStats:
-        return RunStats(s.rounds_max, s.rounds_mean, s.rows_total, s.ms_total, s.launches)
+        return RunStats(s.rounds_max, s.rounds_mean, s.rows_total, s.ms_total, s.launches, s.rows_verified)
 
     def sample(self):
         torch = self._torch

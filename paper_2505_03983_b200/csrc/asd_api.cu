@@ -215,6 +215,7 @@ asd_status asd_create(const asd_config* cfg, void* cuda_stream, asd_ctx** out) {
   if (cfg->K < 1) return bad(ASD_ERR_INVALID_ARG, "K must be >= 1");
   if (cfg->window < 1 || cfg->window > kMaxWindow) return bad(ASD_ERR_INVALID_ARG, "window must be in 1..64");
   if (cfg->max_chains < 1) return bad(ASD_ERR_INVALID_ARG, "max_chains must be >= 1");
+  if (cfg->flags & ~ASD_FLAG_DEBUG_ALL_SLOTS) return bad(ASD_ERR_INVALID_ARG, "unknown flag");
   if (!cfg->t) return bad(ASD_ERR_INVALID_ARG, "t must not be NULL");
   if (!(cfg->t[0] >= 0.0)) return bad(ASD_ERR_INVALID_ARG, "t[0] must be >= 0");
   for (int i = 0; i < cfg->K; ++i) {
@@ -266,6 +267,7 @@ asd_status asd_create(const asd_config* cfg, void* cuda_stream, asd_ctx** out) {
   c->max_chains = cfg->max_chains;
   c->kind = D.kind;
   c->seed = cfg->seed;
+  c->debug_all_slots = (cfg->flags & ASD_FLAG_DEBUG_ALL_SLOTS) != 0;
   c->stream = static_cast<cudaStream_t>(cuda_stream);
   c->max_rows = (int)((long long)cfg->max_chains * std::max(c->window - 1, 1));
   cudaGetDevice(&c->device);
@@ -474,6 +476,7 @@ static asd_status finish_run(Ctx* c, float* y_out_dev, int32_t* rounds_out_dev, 
     cudaEventElapsedTime(&ms, c->ev0, c->ev1);
     stats->ms_total = ms;
     stats->rows_total = (int64_t)c->counters_host->rows_total;
+    stats->rows_verified = (int64_t)c->counters_host->rows_verified;
     stats->launches = c->launches - launches0;
     stats->rounds_max = 0;
     stats->rounds_mean = 0.0;

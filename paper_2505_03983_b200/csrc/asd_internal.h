@@ -27,7 +27,8 @@ struct RoundCounters {
   int err;                      // device error word: 0, or ASD_ERR_TIMEOUT / ASD_ERR_STATE
   unsigned long long accepted;  // steps advanced this round
   unsigned long long rows_total;  // running total of drift evaluations since reset
-  unsigned long long pad[2];
+  unsigned long long rows_verified;  // running total of drift rows the verify kernel read since reset
+  unsigned long long pad[1];
 };
 
 // Per-step fp32 tables, built on the host in fp64 (asd_create).
@@ -106,6 +107,7 @@ struct Ctx {
   int n = 0;  // chains of the current reset
   uint64_t chain_base = 0;
   bool have_reset = false;
+  bool debug_all_slots = false;  // ASD_FLAG_DEBUG_ALL_SLOTS: the verify kernel evaluates every window slot
   // device arrays
   float* y = nullptr;        // [max_chains, d]
   int* a = nullptr;          // [max_chains]

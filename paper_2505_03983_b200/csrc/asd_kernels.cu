@@ -194,9 +194,11 @@ void launch_prep(Ctx* c, int window) {
 // ---------------------------------------------------------------------------------------------
 // Draft (Algorithm 1, proposal loop): y^_{a+k} = y^_{a+k-1} + eta v_a + sigma xi_{a+k} for
 // k = 1..w-1 (the last proposal sample is only needed when the whole window is accepted and is
-// rebuilt by the verify kernel).  One thread owns 4 dims of one chain and walks the window, so the
-// "prefix sum" of the paper is a register recurrence.  Writes the fp32 points and, for the
-// network denoiser, its bf16 input rows.
+// rebuilt by the verify kernel).  A block owns 128 dims of one chain.  The noise of all window
+// slots is generated in parallel (thread = 4 dims x one slot in eight) into shared memory; the
+// "prefix sum" of the paper is then a short serial recurrence over the slots by one warp, in exactly
+// the order of Eq. 7 (so window 1 and the sequential sampler agree bit for bit); finally all threads
+// write the fp32 points and, for the network denoiser, its bf16 input rows.
 // ---------------------------------------------------------------------------------------------
 struct DraftArgs {
   int d, K, window, nq, vec;
@@ -219,7 +221,11 @@ struct DraftArgs {
   const __nv_bfloat16* temb;
 };
 
-__global__ void __launch_bounds__(256) draft_kernel(const DraftArgs A) {
+constexpr int kDraftQ = 32;       // float4 groups (= 128 dims) per block
+constexpr int kDraftThreads = 256;
+
+__global__ void __launch_bounds__(kDraftThreads) draft_kernel(const DraftArgs A) {
+  __shared__ float4 s_pt[kMaxWindow - 1][kDraftQ];  // noise, then drafted points, per slot
   const int p = blockIdx.y;
   if (p >= A.cnt->n_active) return;
   const int j = A.act[p];
@@ -227,18 +233,31 @@ __global__ void __launch_bounds__(256) draft_kernel(const DraftArgs A) {
   const int w = min(A.window, A.K - a);
   const int row0 = A.row_off[p];
   const uint32_t chain = (uint32_t)(A.chain_base + (uint64_t)j);
-  const int q = blockIdx.x * blockDim.x + threadIdx.x;
-  if (q < A.nq) {
+  const int ql = threadIdx.x & (kDraftQ - 1), ks = threadIdx.x / kDraftQ;
+  constexpr int kSlotLanes = kDraftThreads / kDraftQ;
+  const int q = blockIdx.x * kDraftQ + ql;
+  const bool q_ok = q < A.nq;
+  if (q_ok)
+    for (int k = 1 + ks; k < w; k += kSlotLanes) s_pt[k - 1][ql] = xi4((uint32_t)q, (uint32_t)(a + k), chain, A.keys);
+  __syncthreads();
+  if (ks == 0 && q_ok) {
     float4 yh = load4(A.y + (size_t)j * A.d, q, A.d, A.vec);
     const float4 v = load4(A.v + (size_t)p * A.d, q, A.d, A.vec);
     for (int k = 1; k < w; ++k) {
       const int i = a + k - 1;  // step i -> i+1 uses eta_i, sigma_{i+1}, xi_{i+1}
       const float eta = A.tab.eta[i], sig = A.tab.sig[i];
-      const float4 xi = xi4((uint32_t)q, (uint32_t)(i + 1), chain, A.keys);
+      const float4 xi = s_pt[k - 1][ql];
       yh.x = fmaf(sig, xi.x, fmaf(eta, v.x, yh.x));
       yh.y = fmaf(sig, xi.y, fmaf(eta, v.y, yh.y));
       yh.z = fmaf(sig, xi.z, fmaf(eta, v.z, yh.z));
       yh.w = fmaf(sig, xi.w, fmaf(eta, v.w, yh.w));
+      s_pt[k - 1][ql] = yh;
+    }
+  }
+  __syncthreads();
+  if (q_ok) {
+    for (int k = 1 + ks; k < w; k += kSlotLanes) {
+      const float4 yh = s_pt[k - 1][ql];
       const int row = row0 + k - 1;
       store4(A.Yhat + (size_t)row * A.d, q, A.d, A.vec, yh);
       if (A.X) {
@@ -259,25 +278,27 @@ __global__ void __launch_bounds__(256) draft_kernel(const DraftArgs A) {
           if (b + 3 < A.d) xr[3] = __float2bfloat16_rn(ci * yh.w);
         }
       }
-      if (q == 0) {
-        A.row_step[row] = a + k;
-        A.row_slot[row] = j;
-      }
     }
   }
-  // conditioning, time embedding and zero padding of the network input rows
-  if (A.X && blockIdx.x == 0) {
-    const int extra = A.in_pad - A.d;
-    for (int k = 1; k < w; ++k) {
-      const int row = row0 + k - 1;
-      __nv_bfloat16* xr = A.X + (size_t)row * A.in_pad + A.d;
-      for (int e = threadIdx.x; e < extra; e += blockDim.x) {
-        __nv_bfloat16 val = __float2bfloat16_rn(0.f);
-        if (e < A.d_cond)
-          val = A.cond[(size_t)j * A.d_cond + e];
-        else if (e < A.d_cond + A.d_temb)
-          val = A.temb[(size_t)(a + k) * A.d_temb + (e - A.d_cond)];
-        xr[e] = val;
+  if (blockIdx.x == 0) {
+    for (int k = 1 + (int)threadIdx.x; k < w; k += kDraftThreads) {
+      A.row_step[row0 + k - 1] = a + k;
+      A.row_slot[row0 + k - 1] = j;
+    }
+    // conditioning, time embedding and zero padding of the network input rows
+    if (A.X) {
+      const int extra = A.in_pad - A.d;
+      for (int k = 1; k < w; ++k) {
+        const int row = row0 + k - 1;
+        __nv_bfloat16* xr = A.X + (size_t)row * A.in_pad + A.d;
+        for (int e = threadIdx.x; e < extra; e += blockDim.x) {
+          __nv_bfloat16 val = __float2bfloat16_rn(0.f);
+          if (e < A.d_cond)
+            val = A.cond[(size_t)j * A.d_cond + e];
+          else if (e < A.d_cond + A.d_temb)
+            val = A.temb[(size_t)(a + k) * A.d_temb + (e - A.d_cond)];
+          xr[e] = val;
+        }
       }
     }
   }
@@ -312,25 +333,29 @@ void launch_draft(Ctx* c, int window) {
     A.cond = c->mlp.cond;
     A.temb = c->mlp.temb;
   }
-  const int threads = A.nq >= 256 ? 256 : (A.nq >= 128 ? 128 : 64);
-  dim3 grid((A.nq + threads - 1) / threads, c->n);
-  draft_kernel<<<grid, threads, 0, c->stream>>>(A);
+  dim3 grid((A.nq + kDraftQ - 1) / kDraftQ, c->n);
+  draft_kernel<<<grid, kDraftThreads, 0, c->stream>>>(A);
   c->launches++;
 }
 
 // ---------------------------------------------------------------------------------------------
 // Verify + resample + advance (Algorithm 2, Algorithm 3, advance step of Algorithm 1).
-// One block per active chain.  Phase 1: one warp per window slot k >= 2 regenerates xi_{a+k},
-// reads the drift g_{k-1} at the drafted point once (coalesced float4) and reduces
+// One block per active chain.  The block walks the window slots k = 2, 3, ... in order, a few slots at
+// a time (one or two warps per slot); for each slot its warps regenerate xi_{a+k}, read the drift
+// g_{k-1} at the drafted point once (coalesced float4) and reduce
 //   <xi, delta>, |delta|^2, delta = v_a - g_{k-1}      (m^ - m = eta delta)
-// over d with warp shuffles; ln ratio = -(eta/sigma) <xi, delta> - (eta^2 / 2 sigma^2) |delta|^2.
-// Phase 2: a ballot over the accept bits gives the all-accepted prefix length n.
-// Phase 3: the block writes the new state: the reflected sample at the first rejected slot
+// over d (warp shuffles, then a fixed-order sum of the warps' partials that every thread repeats, so
+// all threads reach the same decision without a second barrier);
+//   ln ratio = -(eta/sigma) <xi, delta> - (eta^2 / 2 sigma^2) |delta|^2,  accept iff ln u <= min(0, ln ratio).
+// The Verifier needs only the end of the all-accepted prefix, so the walk stops after the group that
+// holds the first rejected slot: drifts beyond it are never read (all_slots != 0 keeps going, for the
+// diagnostics).
+// Then the block writes the new state: the reflected sample at the first rejected slot
 //   y = y^_n + eta g_n + sigma (xi - 2 delta <delta, xi> / |delta|^2)
 // or, if everything was accepted, the last proposal sample y^_w.
 // ---------------------------------------------------------------------------------------------
 struct VerifyArgs {
-  int d, K, window, nq, vec, use_u;
+  int d, K, window, nq, vec, use_u, all_slots, wps;
   PhiloxKeys keys;
   uint64_t chain_base;
   RoundCounters* cnt;
@@ -348,10 +373,11 @@ struct VerifyArgs {
   int* acc_len;
 };
 
+constexpr int kVerifyMaxWarps = 8;
+
 __global__ void __launch_bounds__(256) verify_kernel(const VerifyArgs A) {
-  __shared__ float s_dot[kMaxWindow + 1], s_nrm[kMaxWindow + 1];
-  __shared__ int s_acc[kMaxWindow + 1];
-  __shared__ int s_n;
+  __shared__ float s_part[2][kVerifyMaxWarps][2][kVerifyMaxWarps];  // [group parity][slot][dot | nrm][warp of team]
+  __shared__ float s_lu[kMaxWindow + 1];
   const int p = blockIdx.x;
   if (p >= A.cnt->n_active) return;
   const int j = A.act[p];
@@ -361,70 +387,104 @@ __global__ void __launch_bounds__(256) verify_kernel(const VerifyArgs A) {
   const uint32_t chain = (uint32_t)(A.chain_base + (uint64_t)j);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
   const float* vrow = A.v + (size_t)p * A.d;
+  const float nan = __int_as_float(0x7fc00000);
 
-  if (tid == 0) {
-    // slot 1: proposal mean == target mean, ratio exactly 1 (Lemma 1)
-    s_acc[1] = 1;
-    A.dbg_lr[(size_t)j * A.window] = 0.f;
-    A.dbg_lu[(size_t)j * A.window] = A.use_u ? ln_u((uint32_t)(a + 1), chain, A.keys) : 0.f;
+  // ln u of every slot (one Philox call each), and the diagnostics of slot 1: proposal mean == target
+  // mean, ratio exactly 1 (Lemma 1)
+  for (int k = 1 + tid; k <= w; k += blockDim.x) {
+    const float lu = A.use_u ? ln_u((uint32_t)(a + k), chain, A.keys) : 0.f;
+    s_lu[k] = lu;
+    A.dbg_lu[(size_t)j * A.window + k - 1] = lu;
+    A.dbg_lr[(size_t)j * A.window + k - 1] = k == 1 ? 0.f : nan;
   }
-  for (int k = 2 + warp; k <= w; k += nwarps) {
-    const float* grow = A.G + (size_t)(row0 + k - 2) * A.d;
+  __syncthreads();
+
+  // Slots are taken in groups of S = nwarps / wps; a team of wps warps reduces one slot.
+  const int wps = A.wps, S = nwarps / wps;
+  const int sw = warp / wps, wl = warp - sw * wps;
+  const int tslot = wl * 32 + lane, team = wps * 32;
+  int n = w;                  // accepted prefix length; w = no rejection seen
+  float rej_dot = 0.f, rej_nrm = 1.f;
+  int par = 0, rows_read = 0;
+  for (int k0 = 2; k0 <= w; k0 += S, par ^= 1) {
+    const int k = k0 + sw;
+    rows_read = min(k0 + S - 1, w) - 1;
     float dot = 0.f, nrm = 0.f;
-    for (int q = lane; q < A.nq; q += 32) {
-      const float4 v = load4(vrow, q, A.d, A.vec);
-      const float4 g = load4(grow, q, A.d, A.vec);
-      const float4 xi = xi4((uint32_t)q, (uint32_t)(a + k), chain, A.keys);
-      float4 dl = make_float4(v.x - g.x, v.y - g.y, v.z - g.z, v.w - g.w);
-      if (!A.vec) {  // ragged tail: dims >= d contribute nothing
-        const int b = 4 * q;
-        if (b + 1 >= A.d) dl.y = 0.f;
-        if (b + 2 >= A.d) dl.z = 0.f;
-        if (b + 3 >= A.d) dl.w = 0.f;
+    if (k <= w) {
+      const float* grow = A.G + (size_t)(row0 + k - 2) * A.d;
+      // four float4 groups per thread at a time: all their loads are issued before the first use
+      for (int q0 = tslot; q0 < A.nq; q0 += 4 * team) {
+        float4 vv[4], gg[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const int q = q0 + u * team;
+          if (q < A.nq) {
+            vv[u] = load4(vrow, q, A.d, A.vec);
+            gg[u] = load4(grow, q, A.d, A.vec);
+          }
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const int q = q0 + u * team;
+          if (q < A.nq) {
+            const float4 xi = xi4((uint32_t)q, (uint32_t)(a + k), chain, A.keys);
+            float4 dl = make_float4(vv[u].x - gg[u].x, vv[u].y - gg[u].y, vv[u].z - gg[u].z, vv[u].w - gg[u].w);
+            if (!A.vec) {  // ragged tail: dims >= d contribute nothing
+              const int b = 4 * q;
+              if (b + 1 >= A.d) dl.y = 0.f;
+              if (b + 2 >= A.d) dl.z = 0.f;
+              if (b + 3 >= A.d) dl.w = 0.f;
+            }
+            dot = fmaf(xi.x, dl.x, dot);
+            dot = fmaf(xi.y, dl.y, dot);
+            dot = fmaf(xi.z, dl.z, dot);
+            dot = fmaf(xi.w, dl.w, dot);
+            nrm = fmaf(dl.x, dl.x, nrm);
+            nrm = fmaf(dl.y, dl.y, nrm);
+            nrm = fmaf(dl.z, dl.z, nrm);
+            nrm = fmaf(dl.w, dl.w, nrm);
+          }
+        }
       }
-      dot = fmaf(xi.x, dl.x, dot);
-      dot = fmaf(xi.y, dl.y, dot);
-      dot = fmaf(xi.z, dl.z, dot);
-      dot = fmaf(xi.w, dl.w, dot);
-      nrm = fmaf(dl.x, dl.x, nrm);
-      nrm = fmaf(dl.y, dl.y, nrm);
-      nrm = fmaf(dl.z, dl.z, nrm);
-      nrm = fmaf(dl.w, dl.w, nrm);
     }
     dot = warp_sum(dot);
     nrm = warp_sum(nrm);
     if (lane == 0) {
-      const int i = a + k - 1;
-      const float lr = -A.tab.c1[i] * dot - A.tab.c2[i] * nrm;
-      const float lu = ln_u((uint32_t)(a + k), chain, A.keys);
-      s_dot[k] = dot;
-      s_nrm[k] = nrm;
-      s_acc[k] = (lu <= fminf(0.f, lr)) || (nrm == 0.f);
-      A.dbg_lr[(size_t)j * A.window + k - 1] = lr;
-      A.dbg_lu[(size_t)j * A.window + k - 1] = lu;
+      s_part[par][sw][0][wl] = dot;
+      s_part[par][sw][1][wl] = nrm;
     }
+    __syncthreads();
+    // every thread walks the group's slots in order and so reaches the same decision
+    bool stop = false;
+    for (int s2 = 0; s2 < S && k0 + s2 <= w; ++s2) {
+      float d2 = 0.f, n2 = 0.f;
+      for (int x = 0; x < wps; ++x) {
+        d2 += s_part[par][s2][0][x];
+        n2 += s_part[par][s2][1][x];
+      }
+      const int kk = k0 + s2, i = a + kk - 1;
+      const float lr = -A.tab.c1[i] * d2 - A.tab.c2[i] * n2;
+      const bool acc = (s_lu[kk] <= fminf(0.f, lr)) || (n2 == 0.f);
+      if (tid == 0) A.dbg_lr[(size_t)j * A.window + kk - 1] = lr;
+      if (!acc && n == w) {
+        n = kk - 1;
+        rej_dot = d2;
+        rej_nrm = n2;
+        if (!A.all_slots) {
+          stop = true;
+          break;
+        }
+      }
+    }
+    if (stop) break;
   }
-  __syncthreads();
-  if (warp == 0) {
-    // first rejected slot: ballot over slots 1..32 and 33..64
-    const int k_lo = lane + 1, k_hi = lane + 33;
-    const unsigned rej_lo = __ballot_sync(0xffffffffu, k_lo <= w && !s_acc[k_lo]);
-    const unsigned rej_hi = __ballot_sync(0xffffffffu, k_hi <= w && !s_acc[k_hi]);
-    int n = w;
-    if (rej_lo)
-      n = __ffs(rej_lo) - 1;  // slot index of first reject is ffs, prefix length is one less
-    else if (rej_hi)
-      n = 32 + __ffs(rej_hi) - 1;
-    if (lane == 0) s_n = n;
-  }
-  __syncthreads();
-  const int n = s_n;
+
   float* yrow = A.y + (size_t)j * A.d;
   if (n < w) {
     // reject at slot n + 1: target mean m = y^_n + eta g_n, reflected noise
     const int i = a + n;
     const float eta = A.tab.eta[i], sig = A.tab.sig[i];
-    const float coef = 2.f * s_dot[n + 1] / s_nrm[n + 1];
+    const float coef = 2.f * rej_dot / rej_nrm;
     const float* base = A.Yhat + (size_t)(row0 + n - 1) * A.d;  // n >= 1 always
     const float* grow = A.G + (size_t)(row0 + n - 1) * A.d;
     for (int q = tid; q < A.nq; q += blockDim.x) {
@@ -462,6 +522,7 @@ __global__ void __launch_bounds__(256) verify_kernel(const VerifyArgs A) {
     A.rounds[j] += 1;
     A.acc_len[j] = n;
     atomicAdd(&A.cnt->accepted, (unsigned long long)adv);
+    atomicAdd(&A.cnt->rows_verified, (unsigned long long)rows_read);
     if (a + adv < A.K) atomicAdd(&A.cnt->n_active_after, 1);
   }
 }
@@ -475,6 +536,7 @@ void launch_verify(Ctx* c, int window, bool use_u) {
   A.nq = (c->d + 3) / 4;
   A.vec = (c->d % 4 == 0);
   A.use_u = use_u;
+  A.all_slots = c->debug_all_slots ? 1 : 0;
   A.keys = make_philox_keys(c->seed);
   A.chain_base = c->chain_base;
   A.cnt = c->counters;
@@ -490,8 +552,9 @@ void launch_verify(Ctx* c, int window, bool use_u) {
   A.dbg_lr = c->dbg_lr;
   A.dbg_lu = c->dbg_lu;
   A.acc_len = c->acc_len;
-  const int threads = (A.nq >= 256 || window > 4) ? 256 : 64;
-  verify_kernel<<<c->n, threads, 0, c->stream>>>(A);
+  // eight warps per chain; a slot is reduced by two warps when a row has >= 512 float4 groups, else by one
+  A.wps = A.nq >= 512 ? 2 : 1;
+  verify_kernel<<<c->n, 256, 0, c->stream>>>(A);
   c->launches++;
 }
 

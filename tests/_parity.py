@@ -61,7 +61,7 @@ def rel_l2(a, b):
 
 
 def lockstep(sampler, wl, n_chains, n_rounds, chain_base=0, check_chains=None, cond=None, log=None,
-             cascade=False):
+             cascade=False, all_slots=False):
     """Runs `n_rounds` rounds on the GPU; before each round the oracle is restarted from the
     GPU's state and must reproduce ln u, ln ratio, the accepted prefix and the new state."""
     g = oden.from_workload(wl)
@@ -69,7 +69,7 @@ def lockstep(sampler, wl, n_chains, n_rounds, chain_base=0, check_chains=None, c
     tol_y, tol_r = tolerances(wl.kind)
     check = list(range(n_chains)) if check_chains is None else list(check_chains)
     sampler.reset(n_chains, chain_base, cond=cond)
-    worst = dict(y=0.0, lr=0.0, lr_over_tol=0.0, lu=0.0, exempt=0, decided=0, rounds=0)
+    worst = dict(y=0.0, lr=0.0, lr_over_tol=0.0, lu=0.0, exempt=0, decided=0, rounds=0, slots=0)
     for r in range(n_rounds):
         a0, y0, _ = [t.cpu().numpy() for t in sampler.get_state()]
         st = sampler.round()
@@ -90,12 +90,19 @@ def lockstep(sampler, wl, n_chains, n_rounds, chain_base=0, check_chains=None, c
                                  sampler.window)
             w = rec.w
             e_lu = np.max(np.abs(lu[j, :w] - rec.ln_u) / np.maximum(1.0, np.abs(rec.ln_u)))
-            d_lr = np.abs(lr[j, :w] - rec.ln_ratio)
+            # the GPU evaluates ln ratio up to and including its first rejected slot (every slot when
+            # the context was created with ASD_FLAG_DEBUG_ALL_SLOTS); the rest is NaN
+            have = ~np.isnan(lr[j, :w])
+            assert np.all(have[:min(int(acc[j]) + 1, w)]), (r, j, acc[j], lr[j, :w])
+            if all_slots:
+                assert np.all(have)
+            d_lr = np.where(have, np.abs(lr[j, :w] - rec.ln_ratio), 0.0)
             tol_lr = ln_ratio_tolerance(wl, sch, rec, cascade)
             e_lr = np.max(d_lr / np.maximum(1.0, np.abs(rec.ln_ratio)))
             worst["lu"] = max(worst["lu"], e_lu)
             worst["lr"] = max(worst["lr"], e_lr)
             worst["lr_over_tol"] = max(worst["lr_over_tol"], float(np.max(d_lr / tol_lr)))
+            worst["slots"] += int(np.sum(have))
             assert e_lu < 1e-5, (r, j, e_lu)
             assert np.all(d_lr < tol_lr), (r, j, d_lr / tol_lr, lr[j, :w], rec.ln_ratio)
             # a decision is compared bit-exactly unless it lies within the margin: 1e-3, or with

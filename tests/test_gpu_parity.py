@@ -116,19 +116,26 @@ def test_lockstep_bench_workload_sampled_chains():
     assert worst["decided"] > 0
 
 # ------------------------------------------------------------------ lock-step rounds
+@pytest.mark.parametrize("all_slots", [False, True])
 @pytest.mark.parametrize("name,chains,rounds", [
     ("cfg1_gmm2d", 16, 60), ("gmm_odd", 9, 30), ("gauss_small", 11, 40), ("cfg2_gauss64", 24, 12),
     ("mlp_tiny", 5, 25), ("mlp_ragged", 37, 8), ("cfg3_policy", 64, 3)])
-def test_lockstep_rounds(name, chains, rounds):
+def test_lockstep_rounds(name, chains, rounds, all_slots):
+    """all_slots=False is the production path (the verify kernel stops at the first rejected slot);
+    all_slots=True makes it evaluate the whole window so every ln ratio is compared."""
+    from paper_2505_03983_b200.binding import FLAG_DEBUG_ALL_SLOTS
     wl = workloads.make(name, chains=chains)
-    with _sampler(wl) as s:
+    with _sampler(wl, flags=FLAG_DEBUG_ALL_SLOTS if all_slots else 0) as s:
         worst = lockstep(s, wl, chains, rounds, chain_base=1000, cond=wl.cond if wl.kind == "mlp" and wl.d_cond else None,
-                         log=_log)
+                         log=_log, all_slots=all_slots)
     assert worst["decided"] > 0
 
 
 def test_lockstep_window_64_and_window_beyond_K():
+    from paper_2505_03983_b200.binding import FLAG_DEBUG_ALL_SLOTS
     wl = workloads.make("gauss_small", K=70, window=64, chains=6)
+    with _sampler(wl, flags=FLAG_DEBUG_ALL_SLOTS) as s:
+        lockstep(s, wl, 6, 10, log=_log, all_slots=True)
     with _sampler(wl) as s:
         lockstep(s, wl, 6, 10, log=_log)
     wl = workloads.make("cfg1_gmm2d", K=20, window=64, chains=4)     # window > K acts like K
