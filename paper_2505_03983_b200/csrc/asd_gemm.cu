@@ -132,6 +132,21 @@ __device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&r)[32]) {
       : "r"(taddr)
       : "memory");
 }
+// 32 lanes x 16 consecutive fp32 columns.
+__device__ __forceinline__ void tc_ld16(uint32_t taddr, uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ float ld_cluster_f32(uint32_t addr) {
+  float v;
+  asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(addr) : "memory");
+  return v;
+}
 __device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
 // ---- CTA-pair (cta_group::2) variants ------------------------------------------------------------
@@ -687,6 +702,181 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
   }
 }
 
+// ---------------------------------------------------------------------------------------------------
+// Skinny kernel for few rows (m <= 256): the product is weight streaming, so the roles of the operands
+// are swapped.  A CTA owns 128 output features: the weight tile W[n0 .. n0+127, k-block] is the MMA's
+// 128-row operand (one 16 KB TMA box per k-block, the shape that streams from HBM at full rate) and the
+// activation rows X[0 .. m_pad-1, k-block] are its narrow operand, so D^T[feature, row] accumulates in
+// tensor memory with no padded MMA rows.  The k range is split over the kSplit CTAs of a cluster so that
+// N/128 x kSplit CTAs keep every SM streaming; each CTA parks its partial accumulator in its own shared
+// memory, then every CTA sums the partials of its share of the rows over distributed shared memory in
+// rank order (a fixed order, so results are reproducible) and applies the fused epilogue, the 32 lanes
+// of a warp writing 32 consecutive features.
+// ---------------------------------------------------------------------------------------------------
+constexpr int kSplit = 4;
+constexpr int kSkinnyMaxStages = 8;
+constexpr int kSkinnyStageBudget = 192 * 1024;
+constexpr int kSkinnyMaxRows = 256;
+
+__host__ __device__ constexpr int skinny_stage_bytes(int m_pad) { return (BM + m_pad) * BK * 2; }
+
+template <int EPI>
+__global__ void __cluster_dims__(kSplit, 1, 1) __launch_bounds__(kGemmThreads, 1)
+gemm_skinny_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x,
+                   const GemmArgs g, const int m_pad, const int S) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t tiles = (raw + 1023u) & ~1023u;
+  const int stage_bytes = skinny_stage_bytes(m_pad);
+  uint8_t* tiles_ptr = smem_raw + (tiles - raw);
+  uint8_t* aux = tiles_ptr + max(S * stage_bytes, m_pad * BM * 4);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(aux);  // full[S], empty[S], acc_full
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(aux + 8 * (2 * S + 1));
+  volatile int* dead = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  const uint32_t bar0 = smem_u32(bars);
+  auto full_bar = [&](int s) { return bar0 + 8u * s; };
+  auto empty_bar = [&](int s) { return bar0 + 8u * (S + s); };
+  const uint32_t accf_bar = bar0 + 8u * (2 * S);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();
+  const int n0 = (blockIdx.x / kSplit) * BM;
+  const int m = min(min(*g.m_dev, g.m_cap), m_pad);
+  const int num_kb = (g.k_dim + BK - 1) / BK;
+  const int per = (num_kb + kSplit - 1) / kSplit;  // k-blocks [kb0, kb1) belong to this rank
+  const int kb0 = min((int)rank * per, num_kb), kb1 = min(kb0 + per, num_kb);
+  const uint32_t tmem_cols = m_pad <= 32 ? 32u : (m_pad <= 64 ? 64u : (m_pad <= 128 ? 128u : 256u));
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < S; ++s) {
+      mbar_init(full_bar(s), 1);
+      mbar_init(empty_bar(s), 1);
+    }
+    mbar_init(accf_bar, 1);
+    *dead = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                 "r"(tmem_cols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ---------------- TMA producer ----------------
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      for (int kb = kb0; kb < kb1; ++kb) {
+        mbar_wait(empty_bar(stage), phase ^ 1u, dead, g.err);
+        const uint32_t sw = tiles + stage * stage_bytes;
+        const uint32_t sx = sw + BM * BK * 2;
+        mbar_expect_tx(full_bar(stage), (uint32_t)stage_bytes);
+        tma_load_2d(sw, &map_w, full_bar(stage), kb * BK, n0);
+        tma_load_2d(sx, &map_x, full_bar(stage), kb * BK, 0);
+        if (++stage == S) {
+          stage = 0;
+          phase ^= 1u;
+        }
+      }
+      drain_after_timeout(dead);
+    }
+  } else if (warp == 1) {
+    // ---------------- MMA issuer ----------------
+    if (lane == 0) {
+      // D fp32, A (weights) and B (activations) bf16, both K-major, M = 128 features, N = m_pad rows
+      const uint32_t idesc =
+          (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(m_pad >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+      int stage = 0;
+      uint32_t phase = 0;
+      for (int kb = kb0; kb < kb1; ++kb) {
+        mbar_wait(full_bar(stage), phase, dead, g.err);
+        tc_fence_after();
+        const uint32_t sw = tiles + stage * stage_bytes;
+        const uint32_t sx = sw + BM * BK * 2;
+        const uint64_t da = smem_desc_sw128(sw), db = smem_desc_sw128(sx);
+#pragma unroll
+        for (int k = 0; k < BK / UMMA_K; ++k)
+          tc_mma_bf16(tmem_base, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), idesc, (kb > kb0 || k > 0) ? 1u : 0u);
+        tc_commit(empty_bar(stage));
+        if (++stage == S) {
+          stage = 0;
+          phase ^= 1u;
+        }
+      }
+      if (kb1 > kb0)
+        tc_commit(accf_bar);
+      else
+        mbar_arrive(accf_bar);  // no k-block of its own: the partial is zero
+    }
+  } else {
+    // ---- park this rank's partial D^T[feature, row] in shared memory as part[row][feature] ----
+    const int quarter = warp & 3;
+    const int feat = quarter * 32 + lane;  // tensor-memory lane = feature within the tile
+    mbar_wait(accf_bar, 0u, dead, g.err);
+    tc_fence_after();
+    float* part = reinterpret_cast<float*>(tiles_ptr);  // the stage buffers are idle now: [m_pad][128] fp32
+    for (int c0 = 0; c0 < m_pad; c0 += 16) {
+      uint32_t r[16];
+      if (kb1 > kb0) {
+        tc_ld16(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)c0, r);
+        tc_wait_ld();
+      } else {
+#pragma unroll
+        for (int e = 0; e < 16; ++e) r[e] = 0u;
+      }
+#pragma unroll
+      for (int e = 0; e < 16; ++e) part[(c0 + e) * BM + feat] = __uint_as_float(r[e]);
+    }
+    tc_fence_before();
+  }
+
+  __syncthreads();
+  __syncwarp();
+  cluster_sync_all();  // every rank's partial is in place
+
+  if (warp >= kEpiWarp0) {
+    const int quarter = warp & 3;
+    const int feat = quarter * 32 + lane;
+    const int n = n0 + feat;
+    if (n < g.n_out) {
+      uint32_t part_of[kSplit];  // the partial buffer sits at the same offset in every CTA of the cluster
+#pragma unroll
+      for (int q = 0; q < kSplit; ++q) part_of[q] = map_to_cta(tiles, (uint32_t)q);
+      const float bias = g.bias[n];
+      for (int row = (int)rank; row < m; row += kSplit) {
+        float acc = 0.f;
+#pragma unroll
+        for (int q = 0; q < kSplit; ++q) acc += ld_cluster_f32(part_of[q] + (uint32_t)((row * BM + feat) * 4));
+        float x = acc + bias;
+        if (EPI == EPI_OUT) {
+          const int step = g.row_step[row];
+          const float ysrc = g.ysrc[(size_t)(g.row_map ? g.row_map[row] : row) * g.n_out + n];
+          g.out_f32[(size_t)row * g.n_out + n] = fmaf(g.c_skip[step], ysrc, g.c_out[step] * x);
+        } else {
+          if (EPI == EPI_HID) x = __bfloat162float(g.resid[(size_t)row * g.ld_h + n]) + silu(x);
+          g.out_bf16[(size_t)row * g.ld_h + n] = __float2bfloat16_rn(x);
+        }
+      }
+    }
+  }
+
+  // no CTA leaves while a peer may still read its partial
+  tc_fence_before();
+  __syncthreads();
+  __syncwarp();
+  cluster_sync_all();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tmem_cols) : "memory");
+  }
+}
+
 // ---- host side --------------------------------------------------------------------------------
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -768,6 +958,36 @@ asd_status launch_gemm_pair_t(Ctx* c, const void* a_ptr, int a_cols, const void*
   return ASD_OK;
 }
 
+template <int EPI>
+asd_status launch_gemm_skinny(Ctx* c, const void* a_ptr, int a_cols, const void* w_ptr, const GemmArgs& g, int m_bound) {
+  const int m_pad = std::max(16, (m_bound + 15) / 16 * 16);
+  CUtensorMap mx, mw;
+  if (!get_tmap(c, a_ptr, g.m_cap, a_cols, m_pad, &mx) || !get_tmap(c, w_ptr, g.n_out, a_cols, BM, &mw)) {
+    c->err = "cuTensorMapEncodeTiled failed";
+    return ASD_ERR_CUDA;
+  }
+  const int stages = std::max(2, std::min(kSkinnyMaxStages, kSkinnyStageBudget / skinny_stage_bytes(m_pad)));
+  const int smem = std::max(stages * skinny_stage_bytes(m_pad), m_pad * BM * 4) + 1024 + 256;
+  static int attr_smem = 0;
+  if (smem > attr_smem) {
+    cudaFuncSetAttribute(gemm_skinny_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    attr_smem = smem;
+  }
+  const int grid = ((g.n_out + BM - 1) / BM) * kSplit;
+  gemm_skinny_kernel<EPI><<<grid, kGemmThreads, smem, c->stream>>>(mw, mx, g, m_pad, stages);
+  c->launches++;
+  return ASD_OK;
+}
+
+// Few rows: weight streaming with swapped operands.  (ASD_GEMM_MODE=cta|pair pins the tiled kernels.)
+bool use_skinny(int m_bound) {
+  static const bool pinned = [] {
+    const char* e = getenv("ASD_GEMM_MODE");
+    return e && (!strcmp(e, "cta") || !strcmp(e, "pair"));
+  }();
+  return !pinned && m_bound <= kSkinnyMaxRows;
+}
+
 // Which kernel and column-tile width serve a [m x k] x [n x k]^T product best.  Model: every SM fills
 // its shared memory from L2 at about 50 bytes per clock and its tensor pipe retires a 128 x 256 x 64
 // block in 512 clocks; a launch takes (waves of tiles) x (k-blocks) x max(fill, math) clocks.
@@ -808,6 +1028,7 @@ GemmPlan plan_gemm(const Ctx* c, int m_bound, int n_out) {
 
 template <int EPI>
 asd_status launch_gemm(Ctx* c, const void* a_ptr, int a_cols, const void* w_ptr, const GemmArgs& g, int m_bound) {
+  if (use_skinny(m_bound)) return launch_gemm_skinny<EPI>(c, a_ptr, a_cols, w_ptr, g, m_bound);
   const GemmPlan p = plan_gemm(c, m_bound, g.n_out);
   if (p.pair) {
     switch (p.bn) {
