@@ -130,7 +130,7 @@ asd_status enqueue_round(Ctx* c, int window, bool use_u, int active_bound) {
 namespace asd {
 ProfScope::ProfScope(Ctx* c_, int phase_) : c(c_ && c_->prof_on ? c_ : nullptr), phase(phase_), l0(0), e0(0) {
   if (!c) return;
-  if (c->ev_used + 2 > c->ev_pool.size()) {
+  while (c->ev_used + 2 > c->ev_pool.size()) {
     for (int i = 0; i < 64; ++i) {
       cudaEvent_t e;
       if (cudaEventCreate(&e) != cudaSuccess) {
@@ -151,9 +151,12 @@ ProfScope::~ProfScope() {
   c->pending.push_back({phase, e0, e0 + 1, (int)(c->launches - l0)});
   c = nullptr;
 }
-void prof_collect(Ctx* c) {
-  if (!c->prof_on && c->pending.empty()) return;
-  for (const auto& p : c->pending) {
+// Folds the first `count` pending event pairs (all of them if count < 0) into c->prof; their events
+// must have completed.
+void prof_collect_some(Ctx* c, long long count) {
+  const size_t n = count < 0 ? c->pending.size() : std::min<size_t>((size_t)count, c->pending.size());
+  for (size_t i = 0; i < n; ++i) {
+    const auto& p = c->pending[i];
     if (p.launches == 0) continue;
     float ms = 0.f;
     if (cudaEventElapsedTime(&ms, c->ev_pool[p.e0], c->ev_pool[p.e1]) == cudaSuccess) {
@@ -161,7 +164,11 @@ void prof_collect(Ctx* c) {
       c->prof[p.phase].launches += p.launches;
     }
   }
-  c->pending.clear();
+  c->pending.erase(c->pending.begin(), c->pending.begin() + n);
+}
+void prof_collect(Ctx* c) {
+  if (!c->prof_on && c->pending.empty()) return;
+  prof_collect_some(c, -1);
   c->ev_used = 0;
 }
 }  // namespace asd
@@ -197,6 +204,9 @@ void asd_destroy(asd_ctx* ctx) {
   cudaStreamSynchronize(c->stream);
   for (void* p : c->dev_allocs) cudaFree(p);
   if (c->counters_host) cudaFreeHost(c->counters_host);
+  if (c->ring_host) cudaFreeHost(c->ring_host);
+  for (cudaEvent_t e : c->ring_ev)
+    if (e) cudaEventDestroy(e);
   if (c->ev0) cudaEventDestroy(c->ev0);
   if (c->ev1) cudaEventDestroy(c->ev1);
   for (cudaEvent_t e : c->ev_pool) cudaEventDestroy(e);
@@ -281,6 +291,12 @@ asd_status asd_create(const asd_config* cfg, void* cuda_stream, asd_ctx** out) {
   if (cudaMallocHost(&c->counters_host, sizeof(RoundCounters)) != cudaSuccess)
     return abandon(fail(c, ASD_ERR_OOM, "pinned allocation failed"));
   memset(c->counters_host, 0, sizeof(RoundCounters));
+  if (cudaMallocHost(&c->ring_host, Ctx::kRing * sizeof(RoundCounters)) != cudaSuccess)
+    return abandon(fail(c, ASD_ERR_OOM, "pinned allocation failed"));
+  memset(c->ring_host, 0, Ctx::kRing * sizeof(RoundCounters));
+  for (int i = 0; i < Ctx::kRing; ++i)
+    if (cudaEventCreateWithFlags(&c->ring_ev[i], cudaEventDisableTiming) != cudaSuccess)
+      return abandon(fail(c, ASD_ERR_CUDA, "event creation failed"));
 
   // ---- per-step tables: fp64 on the host, stored as fp32 -----------------------------------
   const int K = c->K;
@@ -502,22 +518,62 @@ asd_status asd_sample(asd_ctx* ctx, float* y_out_dev, int32_t* rounds_out_dev, a
   if (!c->have_reset) return fail(c, ASD_ERR_STATE, "asd_sample before asd_reset");
   const long long launches0 = c->launches;
   ASD_CUDA(c, cudaEventRecord(c->ev0, c->stream));
+  // The host does not wait for a round before enqueuing the next one: the counters of round r are copied
+  // to a pinned ring slot and read once their event has completed, at most kDepth rounds later.  The
+  // bound on the active chains that sizes the grids is therefore a few rounds old, which is still an
+  // upper bound (chains only finish), and the rounds enqueued after the last chain finished find no
+  // active chain and do nothing.  Theorem 3: the cursor strictly increases, so K rounds always suffice.
+  constexpr int kDepth = 4;
   int active = c->n;
-  // Every chain needs at least ceil(remaining / window) rounds and at most `remaining` (Theorem 3:
-  // the cursor strictly increases); the active count is read back once per round.
-  long long guard = (long long)c->K + 2;
-  while (active > 0 && guard-- > 0) {
-    asd_status st = enqueue_round(c, c->window, true, active);
-    if (st != ASD_OK) return st;
-    st = sync_counters(c);
-    if (st != ASD_OK) return st;
-    active = c->counters_host->n_active_after;
+  long long issued = 0, consumed = 0;
+  const long long max_rounds = (long long)c->K + 2;
+  asd_status deferred = ASD_OK;
+  constexpr size_t kEventsPerRound = 2 * PH_COUNT + 8;  // each ring slot times its phases with its own events
+  size_t prof_pairs[Ctx::kRing] = {};
+  auto consume = [&](bool wait) -> bool {  // false: nothing (more) to read right now
+    const int slot = (int)(consumed % Ctx::kRing);
+    if (wait) {
+      if (cudaEventSynchronize(c->ring_ev[slot]) != cudaSuccess) {
+        deferred = fail(c, ASD_ERR_CUDA, "event synchronisation failed");
+        return false;
+      }
+    } else if (cudaEventQuery(c->ring_ev[slot]) != cudaSuccess) {
+      return false;
+    }
+    const RoundCounters& h = c->ring_host[slot];
+    if (h.err != 0 && deferred == ASD_OK)
+      deferred = fail(c, (asd_status)h.err, "a bounded device-side wait ran out (kernel returned early)");
+    active = h.n_active_after;
     if (c->prof_on) {
-      const long long n1 = c->counters_host->n_active, n2 = c->counters_host->rows2;
+      prof_collect_some(c, (long long)prof_pairs[slot]);
+      const long long n1 = h.n_active, n2 = h.rows2;
       for (int ph : {PH_PREP, PH_PACK, PH_D1_IN, PH_D1_HID, PH_D1_OUT, PH_D1_ANALYTIC, PH_DRAFT, PH_VERIFY})
         c->prof[ph].rows += n1;
       for (int ph : {PH_D2_IN, PH_D2_HID, PH_D2_OUT, PH_D2_ANALYTIC}) c->prof[ph].rows += n2;
     }
+    ++consumed;
+    return true;
+  };
+  while (active > 0 && issued < max_rounds && deferred == ASD_OK) {
+    const int slot = (int)(issued % Ctx::kRing);
+    c->ev_used = (size_t)slot * kEventsPerRound;
+    const size_t pending0 = c->pending.size();
+    asd_status st = enqueue_round(c, c->window, true, active);
+    if (st != ASD_OK) return st;
+    prof_pairs[slot] = c->pending.size() - pending0;
+    ASD_CUDA(c, cudaMemcpyAsync(&c->ring_host[slot], c->counters, sizeof(RoundCounters), cudaMemcpyDeviceToHost, c->stream));
+    ASD_CUDA(c, cudaEventRecord(c->ring_ev[slot], c->stream));
+    ++issued;
+    while (consumed < issued && consume(issued - consumed >= kDepth)) {
+    }
+  }
+  while (consumed < issued && deferred == ASD_OK && consume(true)) {
+  }
+  if (deferred != ASD_OK) {
+    cudaStreamSynchronize(c->stream);
+    cudaMemsetAsync(&c->counters->err, 0, sizeof(int), c->stream);
+    prof_collect(c);
+    return deferred;
   }
   if (active > 0) return fail(c, ASD_ERR_STATE, "chains still active after K rounds");
   return finish_run(c, y_out_dev, rounds_out_dev, stats_host, launches0, true);

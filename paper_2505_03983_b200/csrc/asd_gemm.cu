@@ -744,7 +744,8 @@ gemm_skinny_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
   const int m = min(min(*g.m_dev, g.m_cap), m_pad);
   const int num_kb = (g.k_dim + BK - 1) / BK;
   const int per = (num_kb + kSplit - 1) / kSplit;  // k-blocks [kb0, kb1) belong to this rank
-  const int kb0 = min((int)rank * per, num_kb), kb1 = min(kb0 + per, num_kb);
+  const int kb0 = min((int)rank * per, num_kb);
+  const int kb1 = m > 0 ? min(kb0 + per, num_kb) : kb0;  // no valid row: stream nothing
   const uint32_t tmem_cols = m_pad <= 32 ? 32u : (m_pad <= 64 ? 64u : (m_pad <= 128 ? 128u : 256u));
 
   if (threadIdx.x == 0) {

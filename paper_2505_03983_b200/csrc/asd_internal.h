@@ -126,6 +126,11 @@ struct Ctx {
   int* acc_len = nullptr;    // [max_chains]
   RoundCounters* counters = nullptr;
   RoundCounters* counters_host = nullptr;  // pinned
+  // asd_sample runs ahead of the device: the counters of round r land in ring_host[r % kRing] and
+  // ring_ev[r % kRing] tells when
+  static constexpr int kRing = 8;
+  RoundCounters* ring_host = nullptr;      // pinned [kRing]
+  cudaEvent_t ring_ev[kRing] = {};
   int max_rows = 0;
   Tables tab{};
   GmmParams gmm{};
@@ -154,6 +159,7 @@ struct ProfScope {
   ProfScope(Ctx* c_, int phase_);
   ~ProfScope();
 };
+void prof_collect_some(Ctx* c, long long count);
 void prof_collect(Ctx* c);  // after a stream synchronisation: fold pending event pairs into c->prof
 
 // ---- launchers (asd_kernels.cu) ---------------------------------------------------------
