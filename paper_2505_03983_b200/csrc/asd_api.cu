@@ -1,6 +1,7 @@
 // C ABI of the ASD library: context life cycle, table construction, the host side of the round
 // driver (Algorithm 1's while loop), the sequential sampler (Eq. 7) and the diagnostics.
 #include <math.h>
+#include <stdlib.h>
 #include <stdio.h>
 #include <string.h>
 
@@ -125,6 +126,71 @@ asd_status enqueue_round(Ctx* c, int window, bool use_u, int active_bound) {
   return ASD_OK;
 }
 
+// The bound on the number of active chains that a captured round is built for: the full batch, or the
+// next power of two (so a run needs about log2(n) graphs).
+int bound_bucket(const Ctx* c, int active) {
+  if (active >= c->n) return c->n;
+  int b = 1;
+  while (b < active) b <<= 1;
+  return std::min(b, c->n);
+}
+
+// Enqueues one round on c->stream (which must be the context's private stream): replays the captured
+// graph for this shape, capturing it on first use.
+asd_status launch_round_graph(Ctx* c, int window, bool use_u, int active) {
+  if (active <= 0) return ASD_OK;
+  const int bucket = bound_bucket(c, active);
+  const auto key = std::make_tuple(window, use_u ? 1 : 0, bucket);
+  auto it = c->graphs.find(key);
+  if (it == c->graphs.end()) {
+    const long long l0 = c->launches;
+    ASD_CUDA(c, cudaStreamBeginCapture(c->stream, cudaStreamCaptureModeThreadLocal));
+    const asd_status st = enqueue_round(c, window, use_u, bucket);
+    cudaGraph_t graph = nullptr;
+    const cudaError_t e = cudaStreamEndCapture(c->stream, &graph);
+    const long long captured = c->launches - l0;
+    c->launches = l0;
+    if (st != ASD_OK) {
+      if (graph) cudaGraphDestroy(graph);
+      return st;
+    }
+    if (e != cudaSuccess || !graph) return fail(c, ASD_ERR_CUDA, std::string("stream capture failed: ") + cudaGetErrorString(e));
+    cudaGraphExec_t exec = nullptr;
+    const cudaError_t e2 = cudaGraphInstantiate(&exec, graph, 0);
+    cudaGraphDestroy(graph);
+    if (e2 != cudaSuccess) return fail(c, ASD_ERR_CUDA, std::string("cudaGraphInstantiate: ") + cudaGetErrorString(e2));
+    it = c->graphs.emplace(key, Ctx::RoundGraph{exec, captured}).first;
+  }
+  ASD_CUDA(c, cudaGraphLaunch(it->second.exec, c->stream));
+  c->launches += it->second.launches;
+  return ASD_OK;
+}
+
+// While alive, the context's work goes to its private stream, ordered after what the caller's stream
+// held at construction; the destructor orders the caller's stream after it again.
+struct PrivateStreamScope {
+  Ctx* c;
+  cudaStream_t user;
+  bool on;
+  explicit PrivateStreamScope(Ctx* c_) : c(c_), user(c_->stream), on(false) {
+    if (!c->use_graphs || c->prof_on || !c->gstream) return;
+    if (cudaEventRecord(c->fork_ev, user) != cudaSuccess || cudaStreamWaitEvent(c->gstream, c->fork_ev, 0) != cudaSuccess)
+      return;
+    c->stream = c->gstream;
+    on = true;
+  }
+  ~PrivateStreamScope() {
+    if (!on) return;
+    c->stream = user;
+    cudaEventRecord(c->join_ev, c->gstream);
+    cudaStreamWaitEvent(user, c->join_ev, 0);
+  }
+};
+
+asd_status enqueue_round_any(Ctx* c, bool graphs, int window, bool use_u, int active) {
+  return graphs ? launch_round_graph(c, window, use_u, active) : enqueue_round(c, window, use_u, active);
+}
+
 }  // namespace
 
 namespace asd {
@@ -205,6 +271,13 @@ void asd_destroy(asd_ctx* ctx) {
   for (void* p : c->dev_allocs) cudaFree(p);
   if (c->counters_host) cudaFreeHost(c->counters_host);
   if (c->ring_host) cudaFreeHost(c->ring_host);
+  for (auto& kv : c->graphs) cudaGraphExecDestroy(kv.second.exec);
+  if (c->gstream) {
+    cudaStreamSynchronize(c->gstream);
+    cudaStreamDestroy(c->gstream);
+  }
+  if (c->fork_ev) cudaEventDestroy(c->fork_ev);
+  if (c->join_ev) cudaEventDestroy(c->join_ev);
   for (cudaEvent_t e : c->ring_ev)
     if (e) cudaEventDestroy(e);
   if (c->ev0) cudaEventDestroy(c->ev0);
@@ -291,6 +364,14 @@ asd_status asd_create(const asd_config* cfg, void* cuda_stream, asd_ctx** out) {
   if (cudaMallocHost(&c->counters_host, sizeof(RoundCounters)) != cudaSuccess)
     return abandon(fail(c, ASD_ERR_OOM, "pinned allocation failed"));
   memset(c->counters_host, 0, sizeof(RoundCounters));
+  {
+    const char* e = getenv("ASD_GRAPHS");  // "0" launches every kernel of a round separately
+    c->use_graphs = !(e && e[0] == '0');
+    if (cudaStreamCreateWithFlags(&c->gstream, cudaStreamNonBlocking) != cudaSuccess ||
+        cudaEventCreateWithFlags(&c->fork_ev, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&c->join_ev, cudaEventDisableTiming) != cudaSuccess)
+      return abandon(fail(c, ASD_ERR_CUDA, "stream / event creation failed"));
+  }
   if (cudaMallocHost(&c->ring_host, Ctx::kRing * sizeof(RoundCounters)) != cudaSuccess)
     return abandon(fail(c, ASD_ERR_OOM, "pinned allocation failed"));
   memset(c->ring_host, 0, Ctx::kRing * sizeof(RoundCounters));
@@ -437,6 +518,12 @@ asd_status asd_reset(asd_ctx* ctx, int32_t n_chains, uint64_t chain_id_base, con
   if (chain_id_base + (uint64_t)n_chains > (1ull << 32)) return fail(c, ASD_ERR_INVALID_ARG, "chain ids must stay below 2^32");
   const bool need_cond = c->kind == ASD_DEN_RESMLP_BF16 && c->mlp.d_cond > 0;
   if (need_cond && !cond_dev && n_chains > 0) return fail(c, ASD_ERR_INVALID_ARG, "cond_dev required (d_cond > 0)");
+  if (n_chains != c->n || chain_id_base != c->chain_base) {
+    // the captured rounds hold the batch size and the chain ids in their kernel arguments
+    ASD_CUDA(c, cudaStreamSynchronize(c->gstream));
+    for (auto& kv : c->graphs) cudaGraphExecDestroy(kv.second.exec);
+    c->graphs.clear();
+  }
   c->n = n_chains;
   c->chain_base = chain_id_base;
   const size_t nd = (size_t)n_chains * c->d;
@@ -523,8 +610,11 @@ asd_status asd_sample(asd_ctx* ctx, float* y_out_dev, int32_t* rounds_out_dev, a
   // bound on the active chains that sizes the grids is therefore a few rounds old, which is still an
   // upper bound (chains only finish), and the rounds enqueued after the last chain finished find no
   // active chain and do nothing.  Theorem 3: the cursor strictly increases, so K rounds always suffice.
+  // Unless per-phase timing is on, a round is replayed as one CUDA graph on the context's private stream.
   constexpr int kDepth = 4;
   int active = c->n;
+  {
+  PrivateStreamScope pss(c);
   long long issued = 0, consumed = 0;
   const long long max_rounds = (long long)c->K + 2;
   asd_status deferred = ASD_OK;
@@ -558,7 +648,7 @@ asd_status asd_sample(asd_ctx* ctx, float* y_out_dev, int32_t* rounds_out_dev, a
     const int slot = (int)(issued % Ctx::kRing);
     c->ev_used = (size_t)slot * kEventsPerRound;
     const size_t pending0 = c->pending.size();
-    asd_status st = enqueue_round(c, c->window, true, active);
+    asd_status st = enqueue_round_any(c, pss.on, c->window, true, active);
     if (st != ASD_OK) return st;
     prof_pairs[slot] = c->pending.size() - pending0;
     ASD_CUDA(c, cudaMemcpyAsync(&c->ring_host[slot], c->counters, sizeof(RoundCounters), cudaMemcpyDeviceToHost, c->stream));
@@ -576,6 +666,7 @@ asd_status asd_sample(asd_ctx* ctx, float* y_out_dev, int32_t* rounds_out_dev, a
     return deferred;
   }
   if (active > 0) return fail(c, ASD_ERR_STATE, "chains still active after K rounds");
+  }
   return finish_run(c, y_out_dev, rounds_out_dev, stats_host, launches0, true);
 }
 
@@ -592,9 +683,12 @@ asd_status asd_sequential_ddpm(asd_ctx* ctx, float* y_out_dev, asd_run_stats* st
     for (int v : a) min_a = std::min(min_a, v);
   }
   ASD_CUDA(c, cudaEventRecord(c->ev0, c->stream));
-  for (int i = min_a; i < c->K; ++i) {
-    asd_status st = enqueue_round(c, 1, false, c->n);
-    if (st != ASD_OK) return st;
+  {
+    PrivateStreamScope pss(c);
+    for (int i = min_a; i < c->K; ++i) {
+      asd_status st = enqueue_round_any(c, pss.on, 1, false, c->n);
+      if (st != ASD_OK) return st;
+    }
   }
   return finish_run(c, y_out_dev, nullptr, stats_host, launches0, true);
 }

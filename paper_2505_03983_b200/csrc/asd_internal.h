@@ -138,6 +138,13 @@ struct Ctx {
   MlpParams mlp{};
   std::vector<void*> dev_allocs;
   std::map<std::tuple<const void*, int, int, int>, CUtensorMap> tmaps;
+  // One speculation round captured as a CUDA graph per (window, use_u, bound on active chains); replayed
+  // on a private stream that is forked from and joined to the caller's stream.
+  struct RoundGraph { cudaGraphExec_t exec; long long launches; };
+  std::map<std::tuple<int, int, int>, RoundGraph> graphs;
+  cudaStream_t gstream = nullptr;
+  cudaEvent_t fork_ev = nullptr, join_ev = nullptr;
+  bool use_graphs = true;
   std::string err;
   long long launches = 0;
   cudaEvent_t ev0 = nullptr, ev1 = nullptr;
