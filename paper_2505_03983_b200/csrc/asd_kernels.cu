@@ -194,14 +194,15 @@ void launch_prep(Ctx* c, int window) {
 // ---------------------------------------------------------------------------------------------
 // Draft (Algorithm 1, proposal loop): y^_{a+k} = y^_{a+k-1} + eta v_a + sigma xi_{a+k} for
 // k = 1..w-1 (the last proposal sample is only needed when the whole window is accepted and is
-// rebuilt by the verify kernel).  A block owns 128 dims of one chain.  The noise of all window
-// slots is generated in parallel (thread = 4 dims x one slot in eight) into shared memory; the
-// "prefix sum" of the paper is then a short serial recurrence over the slots by one warp, in exactly
-// the order of Eq. 7 (so window 1 and the sequential sampler agree bit for bit); finally all threads
-// write the fp32 points and, for the network denoiser, its bf16 input rows.
+// rebuilt by the verify kernel).  Two forms with identical arithmetic.  Large batches: one thread owns
+// 4 dims of one chain and walks the window, so the "prefix sum" of the paper is a register recurrence.
+// Small batches: a block owns 128 dims of one chain, the noise of all window slots is generated in
+// parallel (thread = 4 dims x one slot in eight) into shared memory, the recurrence is then a short
+// serial walk over the slots by one warp in exactly the order of Eq. 7, and all threads write the rows.
+// Both write the fp32 points and, for the network denoiser, its bf16 input rows.
 // ---------------------------------------------------------------------------------------------
 struct DraftArgs {
-  int d, K, window, nq, vec;
+  int d, K, window, nq, vec, par;
   PhiloxKeys keys;
   uint64_t chain_base;
   const RoundCounters* cnt;
@@ -224,8 +225,31 @@ struct DraftArgs {
 constexpr int kDraftQ = 32;       // float4 groups (= 128 dims) per block
 constexpr int kDraftThreads = 256;
 
+// fp32 point and (network denoiser) bf16 input of row `row`, slot k, for float4 group q
+__device__ __forceinline__ void draft_store(const DraftArgs& A, int row, int a, int k, int q, float4 yh) {
+  store4(A.Yhat + (size_t)row * A.d, q, A.d, A.vec, yh);
+  if (A.X) {
+    const float ci = A.tab.c_in[a + k];
+    __nv_bfloat16* xr = A.X + (size_t)row * A.in_pad + 4 * q;
+    if (A.vec) {
+      __nv_bfloat162 lo = __floats2bfloat162_rn(ci * yh.x, ci * yh.y);
+      __nv_bfloat162 hi = __floats2bfloat162_rn(ci * yh.z, ci * yh.w);
+      uint2 pk;
+      pk.x = *reinterpret_cast<uint32_t*>(&lo);
+      pk.y = *reinterpret_cast<uint32_t*>(&hi);
+      *reinterpret_cast<uint2*>(xr) = pk;
+    } else {
+      const int b = 4 * q;
+      if (b + 0 < A.d) xr[0] = __float2bfloat16_rn(ci * yh.x);
+      if (b + 1 < A.d) xr[1] = __float2bfloat16_rn(ci * yh.y);
+      if (b + 2 < A.d) xr[2] = __float2bfloat16_rn(ci * yh.z);
+      if (b + 3 < A.d) xr[3] = __float2bfloat16_rn(ci * yh.w);
+    }
+  }
+}
+
 __global__ void __launch_bounds__(kDraftThreads) draft_kernel(const DraftArgs A) {
-  __shared__ float4 s_pt[kMaxWindow - 1][kDraftQ];  // noise, then drafted points, per slot
+  __shared__ float4 s_pt[kMaxWindow - 1][kDraftQ];  // noise, then drafted points, per slot (parallel form)
   const int p = blockIdx.y;
   if (p >= A.cnt->n_active) return;
   const int j = A.act[p];
@@ -233,72 +257,67 @@ __global__ void __launch_bounds__(kDraftThreads) draft_kernel(const DraftArgs A)
   const int w = min(A.window, A.K - a);
   const int row0 = A.row_off[p];
   const uint32_t chain = (uint32_t)(A.chain_base + (uint64_t)j);
-  const int ql = threadIdx.x & (kDraftQ - 1), ks = threadIdx.x / kDraftQ;
-  constexpr int kSlotLanes = kDraftThreads / kDraftQ;
-  const int q = blockIdx.x * kDraftQ + ql;
-  const bool q_ok = q < A.nq;
-  if (q_ok)
-    for (int k = 1 + ks; k < w; k += kSlotLanes) s_pt[k - 1][ql] = xi4((uint32_t)q, (uint32_t)(a + k), chain, A.keys);
-  __syncthreads();
-  if (ks == 0 && q_ok) {
-    float4 yh = load4(A.y + (size_t)j * A.d, q, A.d, A.vec);
-    const float4 v = load4(A.v + (size_t)p * A.d, q, A.d, A.vec);
-    for (int k = 1; k < w; ++k) {
-      const int i = a + k - 1;  // step i -> i+1 uses eta_i, sigma_{i+1}, xi_{i+1}
-      const float eta = A.tab.eta[i], sig = A.tab.sig[i];
-      const float4 xi = s_pt[k - 1][ql];
-      yh.x = fmaf(sig, xi.x, fmaf(eta, v.x, yh.x));
-      yh.y = fmaf(sig, xi.y, fmaf(eta, v.y, yh.y));
-      yh.z = fmaf(sig, xi.z, fmaf(eta, v.z, yh.z));
-      yh.w = fmaf(sig, xi.w, fmaf(eta, v.w, yh.w));
-      s_pt[k - 1][ql] = yh;
-    }
-  }
-  __syncthreads();
-  if (q_ok) {
-    for (int k = 1 + ks; k < w; k += kSlotLanes) {
-      const float4 yh = s_pt[k - 1][ql];
-      const int row = row0 + k - 1;
-      store4(A.Yhat + (size_t)row * A.d, q, A.d, A.vec, yh);
-      if (A.X) {
-        const float ci = A.tab.c_in[a + k];
-        __nv_bfloat16* xr = A.X + (size_t)row * A.in_pad + 4 * q;
-        if (A.vec) {
-          __nv_bfloat162 lo = __floats2bfloat162_rn(ci * yh.x, ci * yh.y);
-          __nv_bfloat162 hi = __floats2bfloat162_rn(ci * yh.z, ci * yh.w);
-          uint2 pk;
-          pk.x = *reinterpret_cast<uint32_t*>(&lo);
-          pk.y = *reinterpret_cast<uint32_t*>(&hi);
-          *reinterpret_cast<uint2*>(xr) = pk;
-        } else {
-          const int b = 4 * q;
-          if (b + 0 < A.d) xr[0] = __float2bfloat16_rn(ci * yh.x);
-          if (b + 1 < A.d) xr[1] = __float2bfloat16_rn(ci * yh.y);
-          if (b + 2 < A.d) xr[2] = __float2bfloat16_rn(ci * yh.z);
-          if (b + 3 < A.d) xr[3] = __float2bfloat16_rn(ci * yh.w);
-        }
+  if (!A.par) {
+    // large batches: one thread owns 4 dims and walks the window; nothing is staged
+    const int q = blockIdx.x * kDraftThreads + threadIdx.x;
+    if (q < A.nq) {
+      float4 yh = load4(A.y + (size_t)j * A.d, q, A.d, A.vec);
+      const float4 v = load4(A.v + (size_t)p * A.d, q, A.d, A.vec);
+      for (int k = 1; k < w; ++k) {
+        const int i = a + k - 1;  // step i -> i+1 uses eta_i, sigma_{i+1}, xi_{i+1}
+        const float eta = A.tab.eta[i], sig = A.tab.sig[i];
+        const float4 xi = xi4((uint32_t)q, (uint32_t)(i + 1), chain, A.keys);
+        yh.x = fmaf(sig, xi.x, fmaf(eta, v.x, yh.x));
+        yh.y = fmaf(sig, xi.y, fmaf(eta, v.y, yh.y));
+        yh.z = fmaf(sig, xi.z, fmaf(eta, v.z, yh.z));
+        yh.w = fmaf(sig, xi.w, fmaf(eta, v.w, yh.w));
+        draft_store(A, row0 + k - 1, a, k, q, yh);
       }
     }
-  }
-  if (blockIdx.x == 0) {
-    for (int k = 1 + (int)threadIdx.x; k < w; k += kDraftThreads) {
-      A.row_step[row0 + k - 1] = a + k;
-      A.row_slot[row0 + k - 1] = j;
+  } else {
+    // small batches: the noise of all slots in parallel, then the recurrence by one warp, then the stores
+    const int ql = threadIdx.x & (kDraftQ - 1), ks = threadIdx.x / kDraftQ;
+    constexpr int kSlotLanes = kDraftThreads / kDraftQ;
+    const int q = blockIdx.x * kDraftQ + ql;
+    const bool q_ok = q < A.nq;
+    if (q_ok)
+      for (int k = 1 + ks; k < w; k += kSlotLanes) s_pt[k - 1][ql] = xi4((uint32_t)q, (uint32_t)(a + k), chain, A.keys);
+    __syncthreads();
+    if (ks == 0 && q_ok) {
+      float4 yh = load4(A.y + (size_t)j * A.d, q, A.d, A.vec);
+      const float4 v = load4(A.v + (size_t)p * A.d, q, A.d, A.vec);
+      for (int k = 1; k < w; ++k) {
+        const int i = a + k - 1;
+        const float eta = A.tab.eta[i], sig = A.tab.sig[i];
+        const float4 xi = s_pt[k - 1][ql];
+        yh.x = fmaf(sig, xi.x, fmaf(eta, v.x, yh.x));
+        yh.y = fmaf(sig, xi.y, fmaf(eta, v.y, yh.y));
+        yh.z = fmaf(sig, xi.z, fmaf(eta, v.z, yh.z));
+        yh.w = fmaf(sig, xi.w, fmaf(eta, v.w, yh.w));
+        s_pt[k - 1][ql] = yh;
+      }
     }
-    // conditioning, time embedding and zero padding of the network input rows
+    __syncthreads();
+    if (q_ok)
+      for (int k = 1 + ks; k < w; k += kSlotLanes) draft_store(A, row0 + k - 1, a, k, q, s_pt[k - 1][ql]);
+  }
+  // row maps, conditioning, time embedding and zero padding: the chain's blocks share the slots
+  for (int k = 1 + (int)blockIdx.x; k < w; k += gridDim.x) {
+    const int row = row0 + k - 1;
+    if (threadIdx.x == 0) {
+      A.row_step[row] = a + k;
+      A.row_slot[row] = j;
+    }
     if (A.X) {
       const int extra = A.in_pad - A.d;
-      for (int k = 1; k < w; ++k) {
-        const int row = row0 + k - 1;
-        __nv_bfloat16* xr = A.X + (size_t)row * A.in_pad + A.d;
-        for (int e = threadIdx.x; e < extra; e += blockDim.x) {
-          __nv_bfloat16 val = __float2bfloat16_rn(0.f);
-          if (e < A.d_cond)
-            val = A.cond[(size_t)j * A.d_cond + e];
-          else if (e < A.d_cond + A.d_temb)
-            val = A.temb[(size_t)(a + k) * A.d_temb + (e - A.d_cond)];
-          xr[e] = val;
-        }
+      __nv_bfloat16* xr = A.X + (size_t)row * A.in_pad + A.d;
+      for (int e = threadIdx.x; e < extra; e += blockDim.x) {
+        __nv_bfloat16 val = __float2bfloat16_rn(0.f);
+        if (e < A.d_cond)
+          val = A.cond[(size_t)j * A.d_cond + e];
+        else if (e < A.d_cond + A.d_temb)
+          val = A.temb[(size_t)(a + k) * A.d_temb + (e - A.d_cond)];
+        xr[e] = val;
       }
     }
   }
@@ -333,7 +352,10 @@ void launch_draft(Ctx* c, int window) {
     A.cond = c->mlp.cond;
     A.temb = c->mlp.temb;
   }
-  dim3 grid((A.nq + kDraftQ - 1) / kDraftQ, c->n);
+  // the staged, slot-parallel form only when one thread per 4 dims would leave the machine mostly idle
+  A.par = (long long)c->n * ((A.nq + kDraftThreads - 1) / kDraftThreads) < 2ll * c->num_sms;
+  const int per_block = A.par ? kDraftQ : kDraftThreads;
+  dim3 grid((A.nq + per_block - 1) / per_block, c->n);
   draft_kernel<<<grid, kDraftThreads, 0, c->stream>>>(A);
   c->launches++;
 }
