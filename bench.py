@@ -30,6 +30,10 @@ if ROOT not in sys.path:
 import workloads  # noqa: E402
 
 DEFAULT_WORKLOAD = "sweep_b512_w64"   # cfg-4 denoiser, 512 chains x window 64, K = 1000 (largest cell)
+# dram__bytes_read.sum + dram__bytes_write.sum of one pass-2 hidden-layer launch of gemm_pair_kernel<256, EPI_HID>
+# at full row count, from the ncu capture summarised in profiles/gemm_pair_hidden_sweep_b512_w16.md; set an entry to
+# None when that kernel changes until the counters are taken again
+NCU_TRAFFIC_BYTES_PER_LAUNCH = {"sweep_b512_w64": 409_598_208 + 244_648_448}
 METRIC = "samples_per_sec"
 UNIT = "samples/s"
 
@@ -120,7 +124,7 @@ def run_reference(args):
     t0 = time.perf_counter()
     rates, desc = [], ""
     for _ in range(args.steps):
-        r, desc = oracle_sample_rate(wl, 10.0, 3)
+        r, desc = oracle_sample_rate(wl, 10.0, 20)
         rates.append(r)
     el = time.perf_counter() - t0
     value = float(np.mean(rates))
@@ -261,7 +265,8 @@ def run_ours(args):
                             "peak_source": peaks["source"] + " (sustained cuBLAS bf16)",
                             "frac_of_burst_peak": ach / peaks["bf16_tflops"],
                             "launches": hid["launches"], "avg_launch_ms": hid["ms"] / max(hid["launches"], 1),
-                            "traffic": None}
+                            "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH.get(wl.name),
+                            "algorithmic_bytes_per_full_launch": int(2 * wl.width * (3 * wl.chains * (wl.window - 1) + wl.width))}
         ver = prof["verify"]
         # bytes the verify kernel has to move: every drift row it reads (it stops after the first
         # rejection, so this is less than the 4 d (w - 1) per chain-round of reading the whole window),
@@ -271,7 +276,10 @@ def run_ours(args):
         line["roofline_verify"] = {"kernel": "verify_kernel", "bound": "hbm", "achieved": vach, "peak": peaks["hbm_gbs"],
                                    "unit": "GB/s", "frac": vach / peaks["hbm_gbs"], "peak_source": peaks["source"],
                                    "launches": ver["launches"], "avg_launch_ms": ver["ms"] / max(ver["launches"], 1),
-                                   "traffic": None}
+                                   "traffic": None,
+                                   "note": "bytes = drift rows actually read (the kernel stops at the first rejection) + "
+                                           "3 rows per chain-round; bound by instruction issue (Philox + Box-Muller per "
+                                           "element) and by the longest accepted prefix, not by HBM"}
     else:
         ver = prof["verify"]
         vbytes = 4.0 * wl.d * (rows_ver + 3 * ver["rows"])
@@ -282,7 +290,7 @@ def run_ours(args):
                             "traffic": None}
     # ---- CPU oracle on a bounded sample (rank 0, N = 1 only) -----------------------------------
     if world == 1 and not args.no_cpu_baseline:
-        rate, desc = oracle_sample_rate(wl, 20.0, 6 if wl.kind == "mlp" and wl.width >= 4096 else 10 ** 9)
+        rate, desc = oracle_sample_rate(wl, 20.0, 10 ** 9)
         try:
             import threadpoolctl
             info = threadpoolctl.threadpool_info()
