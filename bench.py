@@ -311,6 +311,8 @@ def main():
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--sweep", action="store_true",
+                    help="run the 12 cells of the batch x window sweep on the cfg-4 denoiser, one JSON line per cell")
     ap.add_argument("--profile-rounds", type=int, default=0,
                     help="profiling aid: reset, run this many speculation rounds, print nothing timed and exit "
                          "(a short, bounded launch sequence for ncu captures)")
@@ -327,6 +329,10 @@ def main():
             print(json.dumps({"profile_rounds": args.profile_rounds, "workload": wl.name,
                               "last_round": {"active": st.n_active_before, "rows_pass2": st.rows_pass2,
                                              "accepted": st.accepted_total}}))
+    elif args.sweep:
+        for b, w in workloads.SWEEP_CELLS:
+            args.workload, args.no_cpu_baseline = f"sweep_b{b}_w{w}", True
+            run_ours(args)
     elif args.impl == "reference":
         run_reference(args)
     else:
