@@ -220,11 +220,29 @@ def run_ours(args):
     s.reset(n, base, cond=cond_dev)
     _, st_seq = s.sequential_ddpm()
     s.close()
+    # ---- the same workload with per-chain adaptive speculation lengths (ASD_FLAG_ADAPTIVE_WINDOW) ----
+    from paper_2505_03983_b200.binding import FLAG_ADAPTIVE_WINDOW
+    sa = AsdSampler(wl, flags=FLAG_ADAPTIVE_WINDOW)
+    for _ in range(2):
+        sa.reset(n, base, cond=cond_dev)
+        sa.sample()
+    barrier()
+    a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a0.record()
+    ad_rounds, ad_rows = [], 0
+    for _ in range(args.steps):
+        sa.reset(n, base, cond=cond_dev)
+        _, _, st_a = sa.sample()
+        ad_rounds.append(st_a.rounds_mean); ad_rows += st_a.rows_total
+    a1.record()
+    barrier()
+    ms_adapt = a0.elapsed_time(a1)
+    sa.close()
 
-    t = torch.tensor([ms, ms_e2e, st_seq.ms_total, ms_plain], dtype=torch.float64, device="cuda")
+    t = torch.tensor([ms, ms_e2e, st_seq.ms_total, ms_plain, ms_adapt], dtype=torch.float64, device="cuda")
     if dist is not None:
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms, ms_e2e, ms_seq, ms_plain = [float(x) for x in t.cpu()]
+    ms, ms_e2e, ms_seq, ms_plain, ms_adapt = [float(x) for x in t.cpu()]
     if rank != 0:
         if dist is not None:
             dist.destroy_process_group()
@@ -252,6 +270,11 @@ def run_ours(args):
         "sequential_gpu": {"value": n * world / (ms_seq / 1e3), "unit": UNIT, "ms": ms_seq,
                            "wallclock_speedup_asd": (ms_seq) / (ms / args.steps)},
         "without_phase_events": {"value": total / (ms_plain / 1e3), "unit": UNIT, "ms_per_step": ms_plain / args.steps},
+        "adaptive_window": {"value": total / (ms_adapt / 1e3), "unit": UNIT, "ms_per_step": ms_adapt / args.steps,
+                            "rounds_per_sample": float(np.mean(ad_rounds)),
+                            "drift_rows_per_sample_over_K": ad_rows / (args.steps * n * wl.K),
+                            "note": "same workload, every chain picks its speculation length in 2..window from its "
+                                    "own acceptance history (ASD_FLAG_ADAPTIVE_WINDOW); CUDA-graph rounds"},
         "phases_ms": {k: round(v["ms"], 3) for k, v in prof.items() if v["launches"]},
     }
     # ---- roofline of the dominant kernel ----------------------------------------------------

@@ -122,6 +122,21 @@ typedef struct {
  */
 #define ASD_FLAG_DEBUG_ALL_SLOTS 1u
 
+/*
+ * ASD_FLAG_ADAPTIVE_WINDOW: every chain chooses its own speculation length theta_c for the next round
+ * from its own history, between 2 and `window` (the paper fixes theta, Theorem 4 picks it from
+ * K, beta, eta, d; Algorithm 1 is exact for any theta, and a theta that depends only on the chain's past
+ * is adapted to the filtration of its proof).  Rule, in integers so that it is reproducible anywhere:
+ * with p = steps advanced in the round (accepted prefix + the resampled step, or the whole window),
+ *     ema8  <- (ema8 + 8 p) >> 1          (8 x running mean of p, initial value 32)
+ *     theta <- clamp(2 + (3 ema8) / 16, 2, window)     (about 2 + 1.5 x mean; initial min(window, 8))
+ * so a chain that keeps accepting its whole window grows it by half each round and a chain that rejects
+ * early drafts little.  A chain's result still depends only on its id.  asd_sequential_ddpm ignores it.
+ * asd_get_window_state / asd_set_window_state complete the chain state for stop and resume
+ * (device buffers [n] int32 each, any may be NULL; values outside 1..window are clamped when used).
+ */
+#define ASD_FLAG_ADAPTIVE_WINDOW 2u
+
 typedef struct {
   int32_t n_active_before; /* chains with a < K when the round started */
   int32_t n_active_after;
@@ -199,6 +214,8 @@ asd_status asd_sample_host(asd_ctx* ctx, int32_t n_chains, uint64_t chain_id_bas
  */
 asd_status asd_get_state(asd_ctx* ctx, int32_t* a_dev, float* y_dev, int32_t* rounds_dev);
 asd_status asd_set_state(asd_ctx* ctx, const int32_t* a_dev, const float* y_dev, const int32_t* rounds_dev);
+asd_status asd_get_window_state(asd_ctx* ctx, int32_t* window_dev, int32_t* ema8_dev);
+asd_status asd_set_window_state(asd_ctx* ctx, const int32_t* window_dev, const int32_t* ema8_dev);
 
 /*
  * Diagnostics of the last round, indexed by chain position: ln ratio (Algorithm 3) and

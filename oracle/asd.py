@@ -162,6 +162,24 @@ def asd_round(g: Callable, sched: Schedule, seed: int, chain_id: int, slot: int,
 
 
 @dataclasses.dataclass
+class AdaptiveWindow:
+    """Per-chain choice of the speculation length from the chain's own past (an addition of this
+    library: the paper fixes theta; Algorithm 1 is exact for any theta, and a theta that depends only
+    on the past is adapted to the filtration used in the proof of Theorem 3).  Integer rule, so that
+    it can be reproduced exactly: with p = steps advanced in the round,
+        ema8 <- (ema8 + 8 p) >> 1,      theta <- clamp(2 + (3 ema8) // 16, 2, theta_max),
+    starting from ema8 = 32 (theta = min(theta_max, 8))."""
+    theta_max: int
+    ema8: int = 32
+
+    def theta(self) -> int:
+        return max(2, min(self.theta_max, 2 + (3 * self.ema8) // 16))
+
+    def update(self, advanced: int) -> None:
+        self.ema8 = (self.ema8 + 8 * advanced) >> 1
+
+
+@dataclasses.dataclass
 class ChainResult:
     y: np.ndarray
     rounds: int
@@ -176,12 +194,16 @@ class ChainResult:
 
 def asd_sample(g, sched: Schedule, seed: int, chain_id: int, slot: int, theta: int,
                y0=None, d: Optional[int] = None, max_rounds: Optional[int] = None,
-               keep_records: bool = True, a0: int = 0) -> ChainResult:
+               keep_records: bool = True, a0: int = 0, adaptive: bool = False) -> ChainResult:
+    """Algorithm 1.  adaptive=True: theta is the upper limit and every round uses AdaptiveWindow's choice."""
     y = np.zeros(d) if y0 is None else np.asarray(y0, dtype=np.float64).copy()
     a, rounds, rows = a0, 0, 0
     records, traj = [], [y.copy()]
+    policy = AdaptiveWindow(theta) if adaptive else None
     while a < sched.K and (max_rounds is None or rounds < max_rounds):
-        rec = asd_round(g, sched, seed, chain_id, slot, a, y, theta)
+        rec = asd_round(g, sched, seed, chain_id, slot, a, y, policy.theta() if adaptive else theta)
+        if adaptive:
+            policy.update(rec.a_after - rec.a_before)
         rounds += 1
         rows += rec.w                                  # 1 + (w - 1)
         a, y = rec.a_after, rec.y_after

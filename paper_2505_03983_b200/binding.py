@@ -15,7 +15,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 
 EXPORTED_SYMBOLS = [
     "asd_version", "asd_create", "asd_reset", "asd_round", "asd_sample", "asd_sequential_ddpm",
-    "asd_sample_host", "asd_get_state", "asd_set_state", "asd_debug_last_round", "asd_denoise",
+    "asd_sample_host", "asd_get_state", "asd_set_state", "asd_get_window_state", "asd_set_window_state", "asd_debug_last_round", "asd_denoise",
     "asd_set_profiling", "asd_get_profile", "asd_denoise_static", "asd_denoise_static_max_rows",
     "asd_last_error", "asd_destroy",
 ]
@@ -24,6 +24,7 @@ STATUS = {0: "ASD_OK", 1: "ASD_ERR_INVALID_ARG", 2: "ASD_ERR_UNSUPPORTED", 3: "A
           4: "ASD_ERR_CUDA", 5: "ASD_ERR_STATE", 6: "ASD_ERR_TIMEOUT"}
 KIND = {"gmm": 0, "gauss": 1, "mlp": 2}
 FLAG_DEBUG_ALL_SLOTS = 1   # ASD_FLAG_DEBUG_ALL_SLOTS
+FLAG_ADAPTIVE_WINDOW = 2   # ASD_FLAG_ADAPTIVE_WINDOW
 
 
 class AsdError(RuntimeError):
@@ -117,6 +118,8 @@ def load_library():
         "asd_sample_host": [vp, i32, u64, vp, vp, i32, vp, vp, C.POINTER(_RunStats)],
         "asd_get_state": [vp, vp, vp, vp],
         "asd_set_state": [vp, vp, vp, vp],
+        "asd_get_window_state": [vp, vp, vp],
+        "asd_set_window_state": [vp, vp, vp],
         "asd_debug_last_round": [vp, vp, vp, vp],
         "asd_denoise": [vp, i32, vp, vp, vp, vp],
         "asd_denoise_static": [vp, i32, vp, vp, vp, vp],
@@ -290,6 +293,21 @@ class AsdSampler:
         y = None if y is None else y.to(device="cuda", dtype=torch.float32).contiguous()
         rounds = None if rounds is None else rounds.to(device="cuda", dtype=torch.int32).contiguous()
         self._check(self.lib.asd_set_state(self._ctx, _dev_ptr(a), _dev_ptr(y), _dev_ptr(rounds)))
+        torch.cuda.current_stream().synchronize()
+
+    def get_window_state(self):
+        """(speculation length of the next round, 8 x running mean of the steps per round), per chain."""
+        torch = self._torch
+        w, e = self._empty((self.n,), torch.int32), self._empty((self.n,), torch.int32)
+        self._check(self.lib.asd_get_window_state(self._ctx, _dev_ptr(w), _dev_ptr(e)))
+        torch.cuda.current_stream().synchronize()
+        return w, e
+
+    def set_window_state(self, window=None, ema8=None):
+        torch = self._torch
+        window = None if window is None else window.to(device="cuda", dtype=torch.int32).contiguous()
+        ema8 = None if ema8 is None else ema8.to(device="cuda", dtype=torch.int32).contiguous()
+        self._check(self.lib.asd_set_window_state(self._ctx, _dev_ptr(window), _dev_ptr(ema8)))
         torch.cuda.current_stream().synchronize()
 
     def debug_last_round(self):

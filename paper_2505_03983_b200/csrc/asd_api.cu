@@ -19,6 +19,7 @@ struct asd_ctx {
 namespace {
 
 thread_local std::string g_create_error;
+constexpr int kAdaptInitEma8 = 32;
 
 asd_status fail(Ctx* c, asd_status st, const std::string& msg) {
   if (c) c->err = msg;
@@ -298,7 +299,7 @@ asd_status asd_create(const asd_config* cfg, void* cuda_stream, asd_ctx** out) {
   if (cfg->K < 1) return bad(ASD_ERR_INVALID_ARG, "K must be >= 1");
   if (cfg->window < 1 || cfg->window > kMaxWindow) return bad(ASD_ERR_INVALID_ARG, "window must be in 1..64");
   if (cfg->max_chains < 1) return bad(ASD_ERR_INVALID_ARG, "max_chains must be >= 1");
-  if (cfg->flags & ~ASD_FLAG_DEBUG_ALL_SLOTS) return bad(ASD_ERR_INVALID_ARG, "unknown flag");
+  if (cfg->flags & ~(ASD_FLAG_DEBUG_ALL_SLOTS | ASD_FLAG_ADAPTIVE_WINDOW)) return bad(ASD_ERR_INVALID_ARG, "unknown flag");
   if (!cfg->t) return bad(ASD_ERR_INVALID_ARG, "t must not be NULL");
   if (!(cfg->t[0] >= 0.0)) return bad(ASD_ERR_INVALID_ARG, "t[0] must be >= 0");
   for (int i = 0; i < cfg->K; ++i) {
@@ -351,6 +352,7 @@ asd_status asd_create(const asd_config* cfg, void* cuda_stream, asd_ctx** out) {
   c->kind = D.kind;
   c->seed = cfg->seed;
   c->debug_all_slots = (cfg->flags & ASD_FLAG_DEBUG_ALL_SLOTS) != 0;
+  c->adaptive = (cfg->flags & ASD_FLAG_ADAPTIVE_WINDOW) != 0;
   c->stream = static_cast<cudaStream_t>(cuda_stream);
   c->max_rows = (int)((long long)cfg->max_chains * std::max(c->window - 1, 1));
   cudaGetDevice(&c->device);
@@ -414,6 +416,8 @@ asd_status asd_create(const asd_config* cfg, void* cuda_stream, asd_ctx** out) {
   TRY(dev_alloc(c, &c->y, n * d));
   TRY(dev_alloc(c, &c->a, n));
   TRY(dev_alloc(c, &c->rounds, n));
+  TRY(dev_alloc(c, &c->wnd, n));
+  TRY(dev_alloc(c, &c->ema8, n));
   TRY(dev_alloc(c, &c->act, n));
   TRY(dev_alloc(c, &c->row_off, n + 1));
   TRY(dev_alloc(c, &c->step1, n));
@@ -535,6 +539,9 @@ asd_status asd_reset(asd_ctx* ctx, int32_t n_chains, uint64_t chain_id_base, con
   ASD_CUDA(c, cudaMemsetAsync(c->rounds, 0, (size_t)c->max_chains * sizeof(int), c->stream));
   ASD_CUDA(c, cudaMemsetAsync(c->counters, 0, 2 * sizeof(RoundCounters), c->stream));
   launch_fill_int(c, c->acc_len, c->max_chains, -1);
+  // adaptive mode starts every chain at 8 x mean = 32, i.e. a speculation length of min(window, 8)
+  launch_fill_int(c, c->ema8, c->max_chains, kAdaptInitEma8);
+  launch_fill_int(c, c->wnd, c->max_chains, std::max(2, std::min(c->window, 2 + (3 * kAdaptInitEma8) / 16)));
   if (need_cond && n_chains > 0) {
     ASD_CUDA(c, cudaMemcpyAsync(c->cond_f32, cond_dev, (size_t)n_chains * c->mlp.d_cond * sizeof(float),
                                 cudaMemcpyDeviceToDevice, c->stream));
@@ -774,6 +781,24 @@ asd_status asd_set_state(asd_ctx* ctx, const int32_t* a_dev, const float* y_dev,
   if (y_dev) ASD_CUDA(c, cudaMemcpyAsync(c->y, y_dev, (size_t)c->n * c->d * sizeof(float), cudaMemcpyDeviceToDevice, c->stream));
   if (rounds_dev)
     ASD_CUDA(c, cudaMemcpyAsync(c->rounds, rounds_dev, (size_t)c->n * sizeof(int), cudaMemcpyDeviceToDevice, c->stream));
+  return ASD_OK;
+}
+
+asd_status asd_get_window_state(asd_ctx* ctx, int32_t* window_dev, int32_t* ema8_dev) {
+  if (!ctx) return ASD_ERR_INVALID_ARG;
+  Ctx* c = &ctx->c;
+  if (!c->have_reset) return fail(c, ASD_ERR_STATE, "asd_get_window_state before asd_reset");
+  if (window_dev) ASD_CUDA(c, cudaMemcpyAsync(window_dev, c->wnd, (size_t)c->n * sizeof(int), cudaMemcpyDeviceToDevice, c->stream));
+  if (ema8_dev) ASD_CUDA(c, cudaMemcpyAsync(ema8_dev, c->ema8, (size_t)c->n * sizeof(int), cudaMemcpyDeviceToDevice, c->stream));
+  return ASD_OK;
+}
+
+asd_status asd_set_window_state(asd_ctx* ctx, const int32_t* window_dev, const int32_t* ema8_dev) {
+  if (!ctx) return ASD_ERR_INVALID_ARG;
+  Ctx* c = &ctx->c;
+  if (!c->have_reset) return fail(c, ASD_ERR_STATE, "asd_set_window_state before asd_reset");
+  if (window_dev) ASD_CUDA(c, cudaMemcpyAsync(c->wnd, window_dev, (size_t)c->n * sizeof(int), cudaMemcpyDeviceToDevice, c->stream));
+  if (ema8_dev) ASD_CUDA(c, cudaMemcpyAsync(c->ema8, ema8_dev, (size_t)c->n * sizeof(int), cudaMemcpyDeviceToDevice, c->stream));
   return ASD_OK;
 }
 

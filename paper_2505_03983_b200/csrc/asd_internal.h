@@ -107,11 +107,14 @@ struct Ctx {
   int n = 0;  // chains of the current reset
   uint64_t chain_base = 0;
   bool have_reset = false;
+  bool adaptive = false;         // ASD_FLAG_ADAPTIVE_WINDOW
   bool debug_all_slots = false;  // ASD_FLAG_DEBUG_ALL_SLOTS: the verify kernel evaluates every window slot
   // device arrays
   float* y = nullptr;        // [max_chains, d]
   int* a = nullptr;          // [max_chains]
   int* rounds = nullptr;     // [max_chains]
+  int* wnd = nullptr;        // [max_chains] per-chain speculation length of the next round (adaptive mode)
+  int* ema8 = nullptr;       // [max_chains] 8 x running mean of the steps advanced per round (adaptive mode)
   float* cond_f32 = nullptr; // [max_chains, d_cond]
   int* act = nullptr;        // [max_chains] active position -> chain position
   int* row_off = nullptr;    // [max_chains + 1]

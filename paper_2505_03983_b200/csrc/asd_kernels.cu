@@ -99,6 +99,13 @@ __device__ __forceinline__ void store4(float* row, int q, int d, bool vec, float
   if (b + 3 < d) row[b + 3] = val.w;
 }
 
+// Window of chain j this round: its own speculation length (adaptive mode, kept within 1..window) or
+// the common one, cut at the end of the grid (Algorithm 1: b = min(K, a + theta)).
+__device__ __forceinline__ int chain_window(const int* wnd, int j, int window, int K, int a) {
+  const int theta = wnd ? max(1, min(wnd[j], window)) : window;
+  return min(theta, K - a);
+}
+
 __device__ __forceinline__ float warp_sum(float x) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
@@ -109,7 +116,8 @@ __device__ __forceinline__ float warp_sum(float x) {
 // Round driver bookkeeping: compact the chains with a < K into the active list and lay out the
 // pass-2 rows (exclusive scan of w - 1).  One block; n is at most a few tens of thousands.
 // ---------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(1024) prep_kernel(const int* __restrict__ a, int n, int K, int window,
+__global__ void __launch_bounds__(1024) prep_kernel(const int* __restrict__ a, const int* __restrict__ wnd, int n, int K,
+                                                    int window,
                                                     int* __restrict__ act, int* __restrict__ row_off,
                                                     int* __restrict__ step1, int* __restrict__ acc_len,
                                                     RoundCounters* __restrict__ cnt) {
@@ -127,7 +135,7 @@ __global__ void __launch_bounds__(1024) prep_kernel(const int* __restrict__ a, i
     if (j < n) {
       aj = a[j];
       flag = aj < K;
-      rows = flag ? min(window, K - aj) - 1 : 0;
+      rows = flag ? chain_window(wnd, j, window, K, aj) - 1 : 0;
       acc_len[j] = -1;
     }
     // inclusive warp scans
@@ -185,8 +193,11 @@ __global__ void __launch_bounds__(1024) prep_kernel(const int* __restrict__ a, i
   }
 }
 
+// Per-chain speculation lengths apply to speculation rounds only (never to the window-1 steps of Eq. 7).
+static const int* round_windows(const Ctx* c, int window) { return (c->adaptive && window > 1) ? c->wnd : nullptr; }
+
 void launch_prep(Ctx* c, int window) {
-  prep_kernel<<<1, 1024, 0, c->stream>>>(c->a, c->n, c->K, window, c->act, c->row_off, c->step1, c->acc_len,
+  prep_kernel<<<1, 1024, 0, c->stream>>>(c->a, round_windows(c, window), c->n, c->K, window, c->act, c->row_off, c->step1, c->acc_len,
                                          c->counters);
   c->launches++;
 }
@@ -208,6 +219,7 @@ struct DraftArgs {
   const RoundCounters* cnt;
   const int* act;
   const int* a;
+  const int* wnd;  // per-chain speculation length, or null: `window` for every chain
   const int* row_off;
   const float* y;
   const float* v;
@@ -254,7 +266,7 @@ __global__ void __launch_bounds__(kDraftThreads) draft_kernel(const DraftArgs A)
   if (p >= A.cnt->n_active) return;
   const int j = A.act[p];
   const int a = A.a[j];
-  const int w = min(A.window, A.K - a);
+  const int w = chain_window(A.wnd, j, A.window, A.K, a);
   const int row0 = A.row_off[p];
   const uint32_t chain = (uint32_t)(A.chain_base + (uint64_t)j);
   if (!A.par) {
@@ -336,6 +348,7 @@ void launch_draft(Ctx* c, int window) {
   A.cnt = c->counters;
   A.act = c->act;
   A.a = c->a;
+  A.wnd = round_windows(c, window);
   A.row_off = c->row_off;
   A.y = c->y;
   A.v = c->v;
@@ -377,12 +390,14 @@ void launch_draft(Ctx* c, int window) {
 // or, if everything was accepted, the last proposal sample y^_w.
 // ---------------------------------------------------------------------------------------------
 struct VerifyArgs {
-  int d, K, window, nq, vec, use_u, all_slots, wps;
+  int d, K, window, dbg_stride, nq, vec, use_u, all_slots, wps;
   PhiloxKeys keys;
   uint64_t chain_base;
   RoundCounters* cnt;
   const int* act;
   int* a;
+  int* wnd;    // per-chain speculation length (adaptive mode), or null
+  int* ema8;   // 8 x running mean of the steps advanced per round (adaptive mode)
   int* rounds;
   const int* row_off;
   float* y;
@@ -404,7 +419,7 @@ __global__ void __launch_bounds__(256) verify_kernel(const VerifyArgs A) {
   if (p >= A.cnt->n_active) return;
   const int j = A.act[p];
   const int a = A.a[j];
-  const int w = min(A.window, A.K - a);
+  const int w = chain_window(A.wnd, j, A.window, A.K, a);
   const int row0 = A.row_off[p];
   const uint32_t chain = (uint32_t)(A.chain_base + (uint64_t)j);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
@@ -416,8 +431,8 @@ __global__ void __launch_bounds__(256) verify_kernel(const VerifyArgs A) {
   for (int k = 1 + tid; k <= w; k += blockDim.x) {
     const float lu = A.use_u ? ln_u((uint32_t)(a + k), chain, A.keys) : 0.f;
     s_lu[k] = lu;
-    A.dbg_lu[(size_t)j * A.window + k - 1] = lu;
-    A.dbg_lr[(size_t)j * A.window + k - 1] = k == 1 ? 0.f : nan;
+    A.dbg_lu[(size_t)j * A.dbg_stride + k - 1] = lu;
+    A.dbg_lr[(size_t)j * A.dbg_stride + k - 1] = k == 1 ? 0.f : nan;
   }
   __syncthreads();
 
@@ -487,7 +502,7 @@ __global__ void __launch_bounds__(256) verify_kernel(const VerifyArgs A) {
       const int kk = k0 + s2, i = a + kk - 1;
       const float lr = -A.tab.c1[i] * d2 - A.tab.c2[i] * n2;
       const bool acc = (s_lu[kk] <= fminf(0.f, lr)) || (n2 == 0.f);
-      if (tid == 0) A.dbg_lr[(size_t)j * A.window + kk - 1] = lr;
+      if (tid == 0) A.dbg_lr[(size_t)j * A.dbg_stride + kk - 1] = lr;
       if (!acc && n == w) {
         n = kk - 1;
         rej_dot = d2;
@@ -543,6 +558,12 @@ __global__ void __launch_bounds__(256) verify_kernel(const VerifyArgs A) {
     A.a[j] = a + adv;
     A.rounds[j] += 1;
     A.acc_len[j] = n;
+    if (A.wnd) {
+      // next speculation length of this chain: 2 + 1.5 x running mean of the steps it advances per round
+      const int e8 = (A.ema8[j] + 8 * adv) >> 1;
+      A.ema8[j] = e8;
+      A.wnd[j] = max(2, min(A.window, 2 + (3 * e8) / 16));
+    }
     atomicAdd(&A.cnt->accepted, (unsigned long long)adv);
     atomicAdd(&A.cnt->rows_verified, (unsigned long long)rows_read);
     if (a + adv < A.K) atomicAdd(&A.cnt->n_active_after, 1);
@@ -559,6 +580,9 @@ void launch_verify(Ctx* c, int window, bool use_u) {
   A.vec = (c->d % 4 == 0);
   A.use_u = use_u;
   A.all_slots = c->debug_all_slots ? 1 : 0;
+  A.dbg_stride = c->window;
+  A.wnd = const_cast<int*>(round_windows(c, window));
+  A.ema8 = c->ema8;
   A.keys = make_philox_keys(c->seed);
   A.chain_base = c->chain_base;
   A.cnt = c->counters;

@@ -61,7 +61,7 @@ def rel_l2(a, b):
 
 
 def lockstep(sampler, wl, n_chains, n_rounds, chain_base=0, check_chains=None, cond=None, log=None,
-             cascade=False, all_slots=False):
+             cascade=False, all_slots=False, adaptive=False):
     """Runs `n_rounds` rounds on the GPU; before each round the oracle is restarted from the
     GPU's state and must reproduce ln u, ln ratio, the accepted prefix and the new state."""
     g = oden.from_workload(wl)
@@ -72,6 +72,10 @@ def lockstep(sampler, wl, n_chains, n_rounds, chain_base=0, check_chains=None, c
     worst = dict(y=0.0, lr=0.0, lr_over_tol=0.0, lu=0.0, exempt=0, decided=0, rounds=0, slots=0)
     for r in range(n_rounds):
         a0, y0, _ = [t.cpu().numpy() for t in sampler.get_state()]
+        if adaptive:      # every chain has its own speculation length this round
+            theta, ema8 = [t.cpu().numpy() for t in sampler.get_window_state()]
+        else:
+            theta = np.full(n_chains, sampler.window)
         st = sampler.round()
         if st.n_active_before == 0:
             break
@@ -80,14 +84,14 @@ def lockstep(sampler, wl, n_chains, n_rounds, chain_base=0, check_chains=None, c
         assert st.n_active_before == int(np.sum(a0 < wl.K))
         assert st.n_active_after == int(np.sum(a1 < wl.K))
         assert st.accepted_total == int(np.sum(a1 - a0))
-        assert st.rows_pass2 == int(np.sum(np.minimum(sampler.window, wl.K - a0)[a0 < wl.K] - 1))
+        assert st.rows_pass2 == int(np.sum(np.minimum(theta, wl.K - a0)[a0 < wl.K] - 1))
         worst["rounds"] += 1
         for j in check:
             if a0[j] >= wl.K:
                 assert acc[j] == -1 and a1[j] == a0[j] and np.array_equal(y1[j], y0[j])
                 continue
             rec = oasd.asd_round(g, sch, sampler.seed, chain_base + j, j, int(a0[j]), y0[j].astype(np.float64),
-                                 sampler.window)
+                                 int(theta[j]))
             w = rec.w
             e_lu = np.max(np.abs(lu[j, :w] - rec.ln_u) / np.maximum(1.0, np.abs(rec.ln_u)))
             # the GPU evaluates ln ratio up to and including its first rejected slot (every slot when
@@ -119,6 +123,15 @@ def lockstep(sampler, wl, n_chains, n_rounds, chain_base=0, check_chains=None, c
                 e_y = rel_l2(y1[j].astype(np.float64), rec.y_after)
                 worst["y"] = max(worst["y"], e_y)
                 assert e_y < tol_y, (r, j, e_y)
+        if adaptive:      # the integer rule, applied to what the GPU itself advanced
+            theta1, ema81 = [t.cpu().numpy() for t in sampler.get_window_state()]
+            for j in range(n_chains):
+                if a0[j] >= wl.K:
+                    assert theta1[j] == theta[j] and ema81[j] == ema8[j]
+                    continue
+                pol = oasd.AdaptiveWindow(sampler.window, int(ema8[j]))
+                pol.update(int(a1[j] - a0[j]))
+                assert (ema81[j], theta1[j]) == (pol.ema8, pol.theta()), (r, j)
     if log is not None:
         log(f"lockstep {wl.name}: {worst}")
     return worst

@@ -132,6 +132,56 @@ def test_lockstep_rounds(name, chains, rounds, all_slots):
     assert worst["decided"] > 0
 
 
+@pytest.mark.parametrize("name,chains,rounds,window", [("cfg1_gmm2d", 16, 40, 32), ("cfg2_gauss64", 24, 25, 64),
+                                                       ("mlp_ragged", 20, 10, 24), ("cfg3_policy", 32, 4, 64)])
+def test_lockstep_adaptive_window(name, chains, rounds, window):
+    """ASD_FLAG_ADAPTIVE_WINDOW: every chain drafts with its own speculation length; the oracle is run
+    with that length, and the integer rule that updates it is checked against the oracle's."""
+    from paper_2505_03983_b200.binding import FLAG_ADAPTIVE_WINDOW
+    wl = workloads.make(name, chains=chains, window=window)
+    with _sampler(wl, flags=FLAG_ADAPTIVE_WINDOW) as s:
+        worst = lockstep(s, wl, chains, rounds, chain_base=500, cond=wl.cond if wl.kind == "mlp" and wl.d_cond else None,
+                         log=_log, adaptive=True)
+        s.reset(chains, 500, cond=wl.cond if wl.kind == "mlp" and wl.d_cond else None)
+        w, e = s.get_window_state()
+        assert torch.all(w == min(window, 8)) and torch.all(e == 32)
+    assert worst["decided"] > 0
+
+
+def test_adaptive_window_whole_run_and_invariance():
+    """Whole runs with per-chain adaptive windows: chains whose every decision is outside the margin end
+    where the oracle's adaptive run ends, a chain's result does not depend on its batch, and the
+    sequential sampler is unaffected by the flag."""
+    from paper_2505_03983_b200.binding import FLAG_ADAPTIVE_WINDOW
+    wl = workloads.make("cfg2_gauss64", chains=16, K=300, window=64)
+    with _sampler(wl, flags=FLAG_ADAPTIVE_WINDOW) as s:
+        s.reset(16, 40)
+        y, rounds, st = s.sample()
+        s.reset(3, 45)
+        y_part, r_part, _ = s.sample()
+        s.reset(16, 40)
+        y_seq, _ = s.sequential_ddpm()
+    with _sampler(wl) as s0:
+        s0.reset(16, 40)
+        y_seq0, _ = s0.sequential_ddpm()
+        s0.reset(16, 40)
+        _, rounds_fixed, _ = s0.sample()
+    assert torch.equal(y[5:8], y_part) and torch.equal(rounds[5:8], r_part)
+    assert torch.equal(y_seq, y_seq0)
+    g, sch = oden.from_workload(wl), oasd.make_schedule(wl.t)
+    y, rounds = y.cpu().numpy(), rounds.cpu().numpy()
+    compared = 0
+    for j in range(16):
+        res = oasd.asd_sample(g, sch, wl.seed, 40 + j, j, 64, d=wl.d, adaptive=True)
+        if res.min_margin > MARGIN:
+            compared += 1
+            assert rounds[j] == res.rounds
+            assert rel_l2(y[j].astype(np.float64), res.y) < 1e-4
+    _log(f"adaptive cfg2 K=300: rounds mean {rounds.mean():.1f} (fixed window 64: {rounds_fixed.float().mean():.1f}), "
+         f"drift rows {st.rows_total}, compared {compared}")
+    assert compared >= 3
+
+
 def test_lockstep_window_64_and_window_beyond_K():
     from paper_2505_03983_b200.binding import FLAG_DEBUG_ALL_SLOTS
     wl = workloads.make("gauss_small", K=70, window=64, chains=6)

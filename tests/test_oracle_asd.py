@@ -241,3 +241,40 @@ def test_asd_matches_sequential_in_law_on_the_mixture():
     table = table[:, table.sum(0) >= 10]
     assert table.shape[1] >= 2
     assert stats.chi2_contingency(table)[1] > 1e-4
+
+
+def test_adaptive_window_policy_values_and_law():
+    """The per-chain speculation-length rule: hand-computed values, its range, and that Algorithm 1 run
+    with it still samples the Euler chain's law (Theorem 3 holds for any theta; the rule looks only at
+    the chain's past)."""
+    p = asd.AdaptiveWindow(64)
+    assert (p.ema8, p.theta()) == (32, 8)               # 2 + 96 // 16
+    p.update(8)                                         # whole window of 8 accepted: (32 + 64) >> 1 = 48
+    assert (p.ema8, p.theta()) == (48, 11)              # 2 + 144 // 16
+    p.update(1)                                         # rejected at once: (48 + 8) >> 1 = 28
+    assert (p.ema8, p.theta()) == (28, 7)               # 2 + 84 // 16
+    for _ in range(40):
+        p.update(1)
+    assert (p.ema8, p.theta()) == (8, 3)                # floor: a chain always drafts at least 2 + 1
+    for _ in range(40):
+        p.update(p.theta())
+    assert p.theta() == 64                              # ceiling
+    assert asd.AdaptiveWindow(4).theta() == 4 and asd.AdaptiveWindow(2).theta() == 2
+
+    wl = workloads.make("gauss_small", K=24)
+    wl.d = 4
+    wl.mu0, wl.lam = wl.mu0[:4].copy(), wl.lam[:4].copy() * 3
+    wl.Q = np.linalg.qr(wl.Q[:4, :4].astype(np.float64))[0].astype(np.float32)
+    g, sch = den.from_workload(wl), asd.make_schedule(wl.t)
+    Q, lam, mu0 = wl.Q.astype(np.float64), wl.lam.astype(np.float64), wl.mu0.astype(np.float64)
+    mu, P = _euler_gauss_law(np.float32(wl.t).astype(np.float64), mu0, Q, lam)
+    n = 2000
+    res = [asd.asd_sample(g, sch, 5, c, 0, 16, d=4, adaptive=True) for c in range(n)]
+    ya = np.stack([r.y for r in res])
+    windows = np.concatenate([[rec.w for rec in r.records] for r in res[:200]])
+    assert windows.min() >= 1 and windows.max() <= 16 and len(set(windows)) > 3     # it does adapt
+    se = np.sqrt(np.diag(P) / n)
+    assert np.all(np.abs(ya.mean(0) - mu) < 4.5 * se)
+    S = np.cov(ya.T)
+    sd = np.sqrt((np.outer(np.diag(P), np.diag(P)) + P ** 2) / (n - 1))
+    assert np.all(np.abs(S - P) < 4.5 * sd)
