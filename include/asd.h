@@ -254,6 +254,28 @@ asd_status asd_set_profiling(asd_ctx* ctx, int32_t enable);
 asd_status asd_get_profile(asd_ctx* ctx, asd_phase_time* out, int32_t capacity, int32_t* n_out);
 
 /*
+ * DDPM front end (Theorem 1 and the remark after Algorithm 1): from a DDPM noise schedule and the
+ * network's prediction type to the inputs of asd_create.  Host arithmetic only, all pointers host.
+ *   alpha_bar [K+1]: cumulative signal level of the K+1 noise levels the sampler visits, in sampling
+ *                    order, i.e. strictly increasing, inside (0, 1)  (x_level = sqrt(ab) x0 + sqrt(1-ab) eps)
+ *   pred: what the network returns for input x_level - ASD_PRED_X0 (E[x0 | x]), ASD_PRED_EPS, ASD_PRED_V
+ *   map:  ASD_MAP_SL        t = ab / (1 - ab), y = sqrt(t (1 + t)) x, sigma^2 = eta: the Euler chain of the
+ *                           stochastic-localization process that Theorem 1 shows equivalent to the DDPM
+ *         ASD_MAP_ANCESTRAL the DDPM ancestral sampler x_{i+1} = a_i x_i + b_i E[x0 | x_i] + s_i xi itself,
+ *                           written in y_i = x_i / (a_0 .. a_{i-1}) as Eq. 7 with eta_i = b_i / A_{i+1},
+ *                           sigma_{i+1} = s_i / A_{i+1}; s_i^2 = beta~ (large_variance = 0) or beta (1).
+ *                           Meant for the network denoiser (the closed-form drifts read t as SL time).
+ * Outputs: t_out [K+1] and sigma2_out [K] for asd_config, c_in / c_skip / c_out [K] for asd_denoiser,
+ * x_scale [K+1] with x_i = x_scale[i] y_i (start the chain at y_0 = x_0 / x_scale[0]; the DDPM sample
+ * at the last level is x_scale[K] y_K).  Errors: INVALID_ARG.
+ */
+typedef enum { ASD_PRED_X0 = 0, ASD_PRED_EPS = 1, ASD_PRED_V = 2 } asd_pred_kind;
+typedef enum { ASD_MAP_SL = 0, ASD_MAP_ANCESTRAL = 1 } asd_map_kind;
+asd_status asd_ddpm_schedule(int32_t K, const double* alpha_bar, int32_t pred, int32_t map, int32_t large_variance,
+                             double* t_out, double* sigma2_out, float* c_in, float* c_skip, float* c_out,
+                             double* x_scale);
+
+/*
  * asd_denoise_static - the drift of the network denoiser without any device allocation.
  * (The paper has no counterpart: this is a deployment aid of this library.)
  *

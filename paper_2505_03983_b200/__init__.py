@@ -2,5 +2,5 @@
 declared in include/asd.h.  All arithmetic runs in the CUDA library; this package only
 marshals arguments (torch supplies device memory and the stream)."""
 from .binding import (  # noqa: F401
-    AsdError, AsdSampler, RoundStats, RunStats, lib_path, load_library, EXPORTED_SYMBOLS,
+    AsdError, AsdSampler, RoundStats, RunStats, lib_path, load_library, EXPORTED_SYMBOLS, ddpm_schedule,
 )

@@ -16,7 +16,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 EXPORTED_SYMBOLS = [
     "asd_version", "asd_create", "asd_reset", "asd_round", "asd_sample", "asd_sequential_ddpm",
     "asd_sample_host", "asd_get_state", "asd_set_state", "asd_get_window_state", "asd_set_window_state", "asd_debug_last_round", "asd_denoise",
-    "asd_set_profiling", "asd_get_profile", "asd_denoise_static", "asd_denoise_static_max_rows",
+    "asd_set_profiling", "asd_get_profile", "asd_ddpm_schedule", "asd_denoise_static", "asd_denoise_static_max_rows",
     "asd_last_error", "asd_destroy",
 ]
 
@@ -25,6 +25,24 @@ STATUS = {0: "ASD_OK", 1: "ASD_ERR_INVALID_ARG", 2: "ASD_ERR_UNSUPPORTED", 3: "A
 KIND = {"gmm": 0, "gauss": 1, "mlp": 2}
 FLAG_DEBUG_ALL_SLOTS = 1   # ASD_FLAG_DEBUG_ALL_SLOTS
 FLAG_ADAPTIVE_WINDOW = 2   # ASD_FLAG_ADAPTIVE_WINDOW
+
+
+PRED = {"x0": 0, "eps": 1, "v": 2}
+MAP = {"sl": 0, "ancestral": 1}
+
+
+def ddpm_schedule(alpha_bar, pred="eps", mapping="sl", large_variance=False):
+    """asd_ddpm_schedule: dict(t, sigma2, c_in, c_skip, c_out, x_scale) for K = len(alpha_bar) - 1 steps."""
+    lib = load_library()
+    ab = np.ascontiguousarray(alpha_bar, dtype=np.float64)
+    K = len(ab) - 1
+    t, s2, xs = np.empty(K + 1), np.empty(max(K, 0)), np.empty(K + 1)
+    ci, cs, co = (np.empty(max(K, 0), np.float32) for _ in range(3))
+    st = lib.asd_ddpm_schedule(K, _np_ptr(ab), PRED[pred], MAP[mapping], int(large_variance), _np_ptr(t), _np_ptr(s2),
+                               _np_ptr(ci), _np_ptr(cs), _np_ptr(co), _np_ptr(xs))
+    if st != 0:
+        raise AsdError(st, "asd_ddpm_schedule: alpha_bar must be strictly increasing inside (0, 1)")
+    return dict(t=t, sigma2=s2, c_in=ci, c_skip=cs, c_out=co, x_scale=xs)
 
 
 class AsdError(RuntimeError):
@@ -118,6 +136,7 @@ def load_library():
         "asd_sample_host": [vp, i32, u64, vp, vp, i32, vp, vp, C.POINTER(_RunStats)],
         "asd_get_state": [vp, vp, vp, vp],
         "asd_set_state": [vp, vp, vp, vp],
+        "asd_ddpm_schedule": [i32, vp, i32, i32, i32, vp, vp, vp, vp, vp, vp],
         "asd_get_window_state": [vp, vp, vp],
         "asd_set_window_state": [vp, vp, vp],
         "asd_debug_last_round": [vp, vp, vp, vp],

@@ -9,7 +9,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 LIB = os.path.join(HERE, "libasd_b200.so")
-SOURCES = ["asd_api.cu", "asd_kernels.cu", "asd_gemm.cu", "asd_static.cu"]
+SOURCES = ["asd_api.cu", "asd_kernels.cu", "asd_gemm.cu", "asd_static.cu", "asd_schedule.cu"]
 
 
 def _newest(paths):

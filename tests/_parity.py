@@ -61,14 +61,14 @@ def rel_l2(a, b):
 
 
 def lockstep(sampler, wl, n_chains, n_rounds, chain_base=0, check_chains=None, cond=None, log=None,
-             cascade=False, all_slots=False, adaptive=False):
+             cascade=False, all_slots=False, adaptive=False, sigma2=None, y0=None):
     """Runs `n_rounds` rounds on the GPU; before each round the oracle is restarted from the
     GPU's state and must reproduce ln u, ln ratio, the accepted prefix and the new state."""
     g = oden.from_workload(wl)
-    sch = oasd.make_schedule(wl.t)
+    sch = oasd.make_schedule(wl.t, sigma2)
     tol_y, tol_r = tolerances(wl.kind)
     check = list(range(n_chains)) if check_chains is None else list(check_chains)
-    sampler.reset(n_chains, chain_base, cond=cond)
+    sampler.reset(n_chains, chain_base, cond=cond, y0=y0)
     worst = dict(y=0.0, lr=0.0, lr_over_tol=0.0, lu=0.0, exempt=0, decided=0, rounds=0, slots=0)
     for r in range(n_rounds):
         a0, y0, _ = [t.cpu().numpy() for t in sampler.get_state()]

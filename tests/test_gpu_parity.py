@@ -182,6 +182,34 @@ def test_adaptive_window_whole_run_and_invariance():
     assert compared >= 3
 
 
+@pytest.mark.parametrize("mapping,pred", [("sl", "eps"), ("ancestral", "eps"), ("ancestral", "v")])
+def test_ddpm_front_end_chain(mapping, pred):
+    """A chain built by asd_ddpm_schedule (non-uniform steps, explicit variances in the ancestral
+    mapping, c_skip / c_out of an eps- or v-prediction network) started from noise: lock-step rounds
+    and the sequential sampler against the oracle run with the oracle's own copy of the mapping."""
+    import torch as th
+    from oracle import ddpm as oddpm
+    from paper_2505_03983_b200 import ddpm_schedule
+    wl = workloads.make("mlp_tiny", K=40, window=8, chains=6)
+    u = np.linspace(0.0, 1.0, wl.K + 1)
+    ab = 2e-3 + (0.99 - 2e-3) * np.sin(0.5 * np.pi * u) ** 2
+    ours, ref = ddpm_schedule(ab, pred, mapping), oddpm.ddpm_schedule(ab, pred, mapping)
+    rng = np.random.default_rng(2)
+    y0 = (rng.standard_normal((6, wl.d)) / ours["x_scale"][0]).astype(np.float32)
+    wl.t, wl.c_in, wl.c_skip, wl.c_out = ours["t"], ours["c_in"], ours["c_skip"], ours["c_out"]
+    with _sampler(wl, sigma2=ours["sigma2"]) as s:
+        wl.t, wl.c_in, wl.c_skip, wl.c_out = ref["t"], ref["c_in"], ref["c_skip"], ref["c_out"]   # the oracle's copy
+        worst = lockstep(s, wl, 6, 12, chain_base=9, cond=wl.cond, log=_log, sigma2=ref["sigma2"],
+                         y0=th.as_tensor(y0, device="cuda"))
+        s.reset(6, 9, cond=wl.cond, y0=th.as_tensor(y0, device="cuda"))
+        y_seq, _ = s.sequential_ddpm()
+    assert worst["decided"] > 0
+    g, sch = oden.from_workload(wl), oasd.make_schedule(ref["t"], ref["sigma2"])
+    for j in range(6):
+        yr = oasd.sequential_ddpm(g, sch, wl.seed, 9 + j, j, y0=y0[j].astype(np.float64))
+        assert rel_l2(y_seq[j].cpu().numpy().astype(np.float64), yr) < 5e-2
+
+
 def test_lockstep_window_64_and_window_beyond_K():
     from paper_2505_03983_b200.binding import FLAG_DEBUG_ALL_SLOTS
     wl = workloads.make("gauss_small", K=70, window=64, chains=6)
