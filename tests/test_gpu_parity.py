@@ -108,6 +108,17 @@ def test_drift_cfg4_network_rows():
     _log(f"drift cfg4_image rows={n_rows}: max |out - ref| / |network branch| {rel.max():.3e}")
     assert rel.max() < 2.0 ** -7
 
+@pytest.mark.parametrize("name,check,rounds,cascade", [("cfg2_gauss64", [0, 100, 255], 6, False),
+                                                       ("cfg4_image", [0, 13, 31], 3, True)])
+def test_lockstep_full_size_configs_sampled_chains(name, check, rounds, cascade):
+    """cfg2 (256 chains) and cfg4 (32 chains x window 32, the 6-layer width-4096 network) at their full
+    batch sizes; the oracle re-runs a sample of the chains."""
+    wl = workloads.make(name)
+    with _sampler(wl) as s:
+        worst = lockstep(s, wl, wl.chains, rounds, check_chains=check, log=_log, cascade=cascade)
+    assert worst["decided"] > 0
+
+
 def test_lockstep_bench_workload_sampled_chains():
     """The bench's own launch configuration (cfg-4 network, 512 chains x window 64: 32256 drafted rows
     per round) for two rounds; the oracle re-runs a sample of the chains from the GPU's state."""
