@@ -142,9 +142,11 @@ __device__ __forceinline__ void tc_ld16(uint32_t taddr, uint32_t (&r)[16]) {
       : "r"(taddr)
       : "memory");
 }
+// Not volatile and without a memory clobber: the loads of several rows may be in flight together; the
+// cluster barrier that precedes them orders them after the peers' stores.
 __device__ __forceinline__ float ld_cluster_f32(uint32_t addr) {
   float v;
-  asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(addr) : "memory");
+  asm("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(addr));
   return v;
 }
 __device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
@@ -703,7 +705,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
 }
 
 // ---------------------------------------------------------------------------------------------------
-// Skinny kernel for few rows (m <= 256): the product is weight streaming, so the roles of the operands
+// Skinny kernel for few rows (used for m <= 256; gridDim.y walks further blocks of 256 rows): the product is weight streaming, so the roles of the operands
 // are swapped.  A CTA owns 128 output features: the weight tile W[n0 .. n0+127, k-block] is the MMA's
 // 128-row operand (one 16 KB TMA box per k-block, the shape that streams from HBM at full rate) and the
 // activation rows X[0 .. m_pad-1, k-block] are its narrow operand, so D^T[feature, row] accumulates in
@@ -716,7 +718,8 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
 constexpr int kSplit = 4;
 constexpr int kSkinnyMaxStages = 8;
 constexpr int kSkinnyStageBudget = 192 * 1024;
-constexpr int kSkinnyMaxRows = 256;
+constexpr int kSkinnyBlockRows = 256;  // activation rows per CTA (the MMA's N)
+constexpr int kSkinnyMaxRows = 256;    // one row block: at 512 rows the CTA-pair kernel with 128-wide tiles is as fast
 
 __host__ __device__ constexpr int skinny_stage_bytes(int m_pad) { return (BM + m_pad) * BK * 2; }
 
@@ -741,7 +744,8 @@ gemm_skinny_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = cluster_ctarank();
   const int n0 = (blockIdx.x / kSplit) * BM;
-  const int m = min(min(*g.m_dev, g.m_cap), m_pad);
+  const int row0 = blockIdx.y * m_pad;  // this CTA's block of activation rows
+  const int m = max(0, min(min(*g.m_dev, g.m_cap) - row0, m_pad));
   const int num_kb = (g.k_dim + BK - 1) / BK;
   const int per = (num_kb + kSplit - 1) / kSplit;  // k-blocks [kb0, kb1) belong to this rank
   const int kb0 = min((int)rank * per, num_kb);
@@ -779,7 +783,7 @@ gemm_skinny_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
         const uint32_t sx = sw + BM * BK * 2;
         mbar_expect_tx(full_bar(stage), (uint32_t)stage_bytes);
         tma_load_2d(sw, &map_w, full_bar(stage), kb * BK, n0);
-        tma_load_2d(sx, &map_x, full_bar(stage), kb * BK, 0);
+        tma_load_2d(sx, &map_x, full_bar(stage), kb * BK, row0);
         if (++stage == S) {
           stage = 0;
           phase ^= 1u;
@@ -850,18 +854,42 @@ gemm_skinny_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
 #pragma unroll
       for (int q = 0; q < kSplit; ++q) part_of[q] = map_to_cta(tiles, (uint32_t)q);
       const float bias = g.bias[n];
-      for (int row = (int)rank; row < m; row += kSplit) {
-        float acc = 0.f;
+      // rows rank, rank + kSplit, ... of the block, eight at a time: all their loads (partials over
+      // distributed shared memory, residual / state and per-row scalars from global memory) are issued
+      // before the first store, so one memory latency is paid per group instead of per row
+      constexpr int R = 8;
+      for (int lr0 = (int)rank; lr0 < m; lr0 += R * kSplit) {
+        float acc[R], opnd[R], cs[R], co[R];
 #pragma unroll
-        for (int q = 0; q < kSplit; ++q) acc += ld_cluster_f32(part_of[q] + (uint32_t)((row * BM + feat) * 4));
-        float x = acc + bias;
-        if (EPI == EPI_OUT) {
-          const int step = g.row_step[row];
-          const float ysrc = g.ysrc[(size_t)(g.row_map ? g.row_map[row] : row) * g.n_out + n];
-          g.out_f32[(size_t)row * g.n_out + n] = fmaf(g.c_skip[step], ysrc, g.c_out[step] * x);
-        } else {
-          if (EPI == EPI_HID) x = __bfloat162float(g.resid[(size_t)row * g.ld_h + n]) + silu(x);
-          g.out_bf16[(size_t)row * g.ld_h + n] = __float2bfloat16_rn(x);
+        for (int u = 0; u < R; ++u) {
+          const int lr = min(lr0 + u * kSplit, m - 1);  // clamped rows are loaded but not stored
+          const int row = row0 + lr;
+          float a = 0.f;
+#pragma unroll
+          for (int q = 0; q < kSplit; ++q) a += ld_cluster_f32(part_of[q] + (uint32_t)((lr * BM + feat) * 4));
+          acc[u] = a;
+          if (EPI == EPI_OUT) {
+            const int step = g.row_step[row];
+            cs[u] = g.c_skip[step];
+            co[u] = g.c_out[step];
+            opnd[u] = g.ysrc[(size_t)(g.row_map ? g.row_map[row] : row) * g.n_out + n];
+          } else if (EPI == EPI_HID) {
+            opnd[u] = __bfloat162float(g.resid[(size_t)row * g.ld_h + n]);
+          }
+        }
+#pragma unroll
+        for (int u = 0; u < R; ++u) {
+          const int lr = lr0 + u * kSplit;
+          if (lr < m) {
+            const int row = row0 + lr;
+            float x = acc[u] + bias;
+            if (EPI == EPI_OUT) {
+              g.out_f32[(size_t)row * g.n_out + n] = fmaf(cs[u], opnd[u], co[u] * x);
+            } else {
+              if (EPI == EPI_HID) x = opnd[u] + silu(x);
+              g.out_bf16[(size_t)row * g.ld_h + n] = __float2bfloat16_rn(x);
+            }
+          }
         }
       }
     }
@@ -961,7 +989,8 @@ asd_status launch_gemm_pair_t(Ctx* c, const void* a_ptr, int a_cols, const void*
 
 template <int EPI>
 asd_status launch_gemm_skinny(Ctx* c, const void* a_ptr, int a_cols, const void* w_ptr, const GemmArgs& g, int m_bound) {
-  const int m_pad = std::max(16, (m_bound + 15) / 16 * 16);
+  const int m_pad = std::min(kSkinnyBlockRows, std::max(16, (m_bound + 15) / 16 * 16));
+  const int row_blocks = (m_bound + m_pad - 1) / m_pad;
   CUtensorMap mx, mw;
   if (!get_tmap(c, a_ptr, g.m_cap, a_cols, m_pad, &mx) || !get_tmap(c, w_ptr, g.n_out, a_cols, BM, &mw)) {
     c->err = "cuTensorMapEncodeTiled failed";
@@ -974,7 +1003,7 @@ asd_status launch_gemm_skinny(Ctx* c, const void* a_ptr, int a_cols, const void*
     cudaFuncSetAttribute(gemm_skinny_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     attr_smem = smem;
   }
-  const int grid = ((g.n_out + BM - 1) / BM) * kSplit;
+  const dim3 grid(((g.n_out + BM - 1) / BM) * kSplit, row_blocks);
   gemm_skinny_kernel<EPI><<<grid, kGemmThreads, smem, c->stream>>>(mw, mx, g, m_pad, stages);
   c->launches++;
   return ASD_OK;

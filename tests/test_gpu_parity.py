@@ -29,7 +29,7 @@ def _log(msg):
 @pytest.mark.parametrize("name,n_rows", [("cfg1_gmm2d", 100), ("gmm_odd", 57), ("gauss_small", 50),
                                          ("cfg2_gauss64", 300), ("mlp_tiny", 23), ("mlp_ragged", 300),
                                          ("mlp_ragged", 1), ("mlp_ragged", 200), ("cfg3_policy", 17),
-                                         ("cfg3_policy", 256), ("cfg3_policy", 700)])
+                                         ("cfg3_policy", 256), ("cfg3_policy", 400), ("cfg3_policy", 512), ("cfg3_policy", 700)])
 def test_drift_matches_oracle(name, n_rows):
     wl = workloads.make(name)
     rng = np.random.default_rng(5)

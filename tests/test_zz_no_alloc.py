@@ -57,7 +57,10 @@ def test_static_scratch_entry_point_matches_asd_denoise():
             s.denoise(steps, y, slots)
         big = s.denoise_static(steps, y, slots)
         head = s.denoise(steps[:ctx_rows], y[:ctx_rows], slots[:ctx_rows])
-        assert torch.equal(big[:ctx_rows], head) and torch.isfinite(big).all()
+        # a different row count may select a different GEMM kernel (another summation order), so this
+        # comparison uses the tolerance of the drift parity test rather than bit equality
+        assert torch.isfinite(big).all()
+        assert (big[:ctx_rows] - head).abs().max().item() / max(1.0, head.abs().max().item()) < 2e-3
         # beyond the maximum: rejected with a clear error, nothing launched
         st = lib.asd_denoise_static(ctx, max_rows + 1, C.c_void_p(steps.data_ptr()), C.c_void_p(y.data_ptr()),
                                     C.c_void_p(slots.data_ptr()), C.c_void_p(big.data_ptr()))
