@@ -151,6 +151,10 @@ __device__ __forceinline__ float ld_cluster_f32(uint32_t addr) {
 }
 __device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
+// Programmatic dependent launch (no-ops for a kernel launched without that attribute).
+__device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 // ---- CTA-pair (cta_group::2) variants ------------------------------------------------------------
 __device__ __forceinline__ uint32_t cluster_ctarank() {
   uint32_t r;
@@ -718,6 +722,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
 constexpr int kSplit = 4;
 constexpr int kSkinnyMaxStages = 8;
 constexpr int kSkinnyStageBudget = 192 * 1024;
+constexpr int kSkinnySmallBudget = 96 * 1024;  // up to 128 rows: two CTAs (consecutive layers) share an SM
 constexpr int kSkinnyBlockRows = 256;  // activation rows per CTA (the MMA's N)
 constexpr int kSkinnyMaxRows = 256;    // one row block: at 512 rows the CTA-pair kernel with 128-wide tiles is as fast
 
@@ -745,12 +750,15 @@ gemm_skinny_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
   const uint32_t rank = cluster_ctarank();
   const int n0 = (blockIdx.x / kSplit) * BM;
   const int row0 = blockIdx.y * m_pad;  // this CTA's block of activation rows
-  const int m = max(0, min(min(*g.m_dev, g.m_cap) - row0, m_pad));
   const int num_kb = (g.k_dim + BK - 1) / BK;
   const int per = (num_kb + kSplit - 1) / kSplit;  // k-blocks [kb0, kb1) belong to this rank
-  const int kb0 = min((int)rank * per, num_kb);
-  const int kb1 = m > 0 ? min(kb0 + per, num_kb) : kb0;  // no valid row: stream nothing
+  const int kb0 = min((int)rank * per, num_kb), kb1 = min(kb0 + per, num_kb);
   const uint32_t tmem_cols = m_pad <= 32 ? 32u : (m_pad <= 64 ? 64u : (m_pad <= 128 ? 128u : 256u));
+
+  // Programmatic dependent launch: the next kernel of the stream may start its own preamble now (if it was
+  // launched with that attribute); everything here that depends on an earlier kernel comes after
+  // grid_dependency_wait() below.  The weights do not, so their first tiles are fetched before it.
+  grid_launch_dependents();
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < S; ++s) {
@@ -775,9 +783,19 @@ gemm_skinny_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
   if (warp == 0) {
     // ---------------- TMA producer ----------------
     if (lane == 0) {
-      int stage = 0;
-      uint32_t phase = 0;
-      for (int kb = kb0; kb < kb1; ++kb) {
+      // the first min(S, k-blocks) stages are free: weight tiles now, activation tiles once the producer
+      // of the activations has finished
+      const int pre = min(S, kb1 - kb0);
+      for (int i = 0; i < pre; ++i) {
+        mbar_expect_tx(full_bar(i), (uint32_t)stage_bytes);
+        tma_load_2d(tiles + i * stage_bytes, &map_w, full_bar(i), (kb0 + i) * BK, n0);
+      }
+      grid_dependency_wait();
+      for (int i = 0; i < pre; ++i)
+        tma_load_2d(tiles + i * stage_bytes + BM * BK * 2, &map_x, full_bar(i), (kb0 + i) * BK, row0);
+      int stage = pre == S ? 0 : pre;
+      uint32_t phase = pre == S ? 1u : 0u;
+      for (int kb = kb0 + pre; kb < kb1; ++kb) {
         mbar_wait(empty_bar(stage), phase ^ 1u, dead, g.err);
         const uint32_t sw = tiles + stage * stage_bytes;
         const uint32_t sx = sw + BM * BK * 2;
@@ -849,6 +867,8 @@ gemm_skinny_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
     const int quarter = warp & 3;
     const int feat = quarter * 32 + lane;
     const int n = n0 + feat;
+    grid_dependency_wait();  // the row count, the residual and the state come from earlier kernels
+    const int m = max(0, min(min(*g.m_dev, g.m_cap) - row0, m_pad));
     if (n < g.n_out) {
       uint32_t part_of[kSplit];  // the partial buffer sits at the same offset in every CTA of the cluster
 #pragma unroll
@@ -996,7 +1016,8 @@ asd_status launch_gemm_skinny(Ctx* c, const void* a_ptr, int a_cols, const void*
     c->err = "cuTensorMapEncodeTiled failed";
     return ASD_ERR_CUDA;
   }
-  const int stages = std::max(2, std::min(kSkinnyMaxStages, kSkinnyStageBudget / skinny_stage_bytes(m_pad)));
+  const int budget = m_pad <= 128 ? kSkinnySmallBudget : kSkinnyStageBudget;
+  const int stages = std::max(2, std::min(kSkinnyMaxStages, budget / skinny_stage_bytes(m_pad)));
   const int smem = std::max(stages * skinny_stage_bytes(m_pad), m_pad * BM * 4) + 1024 + 256;
   static int attr_smem = 0;
   if (smem > attr_smem) {
@@ -1004,7 +1025,23 @@ asd_status launch_gemm_skinny(Ctx* c, const void* a_ptr, int a_cols, const void*
     attr_smem = smem;
   }
   const dim3 grid(((g.n_out + BM - 1) / BM) * kSplit, row_blocks);
-  gemm_skinny_kernel<EPI><<<grid, kGemmThreads, smem, c->stream>>>(mw, mx, g, m_pad, stages);
+  // Programmatic dependent launch: this kernel may begin (barriers, tensor memory, first weight tiles)
+  // while the previous kernel of the stream is still finishing; it waits for it before it touches
+  // anything that kernel wrote.
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = dim3(kGemmThreads);
+  cfg.dynamicSmemBytes = (size_t)smem;
+  cfg.stream = c->stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  if (cudaLaunchKernelEx(&cfg, gemm_skinny_kernel<EPI>, mw, mx, g, m_pad, stages) != cudaSuccess) {
+    c->err = std::string("skinny GEMM launch failed: ") + cudaGetErrorString(cudaGetLastError());
+    return ASD_ERR_CUDA;
+  }
   c->launches++;
   return ASD_OK;
 }
