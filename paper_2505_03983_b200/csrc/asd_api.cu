@@ -80,7 +80,7 @@ asd_status enqueue_round(Ctx* c, int window, bool use_u, int active_bound) {
   if (active_bound <= 0) return ASD_OK;
   {
     ProfScope ps(c, PH_PREP);
-    launch_prep(c, window);
+    launch_prep(c, whole_batch(c), window);
   }
   RowSet rs1{&c->counters->n_active, active_bound, c->y, c->act, c->step1, c->act};
   RowSet rs2{&c->counters->rows2, active_bound * (window - 1), c->Yhat, nullptr, c->row_step, c->row_slot};
@@ -95,7 +95,7 @@ asd_status enqueue_round(Ctx* c, int window, bool use_u, int active_bound) {
       }
       {
         ProfScope ps(c, PH_DRAFT);
-        launch_draft(c, window);
+        launch_draft(c, whole_batch(c), window, c->v, nullptr);
       }
       {
         ProfScope ps(c, PH_D2_ANALYTIC);
@@ -112,7 +112,7 @@ asd_status enqueue_round(Ctx* c, int window, bool use_u, int active_bound) {
       if (st != ASD_OK) return st;
       {
         ProfScope ps(c, PH_DRAFT);
-        launch_draft(c, window);
+        launch_draft(c, whole_batch(c), window, c->v, nullptr);
       }
       st = mlp_forward(c, rs2, c->G, 1);
       if (st != ASD_OK) return st;
@@ -121,7 +121,7 @@ asd_status enqueue_round(Ctx* c, int window, bool use_u, int active_bound) {
   }
   {
     ProfScope ps(c, PH_VERIFY);
-    launch_verify(c, window, use_u);
+    launch_verify(c, whole_batch(c), window, use_u, c->G, c->v, nullptr);
   }
   ASD_CUDA(c, cudaGetLastError());
   return ASD_OK;

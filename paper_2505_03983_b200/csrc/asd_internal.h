@@ -84,6 +84,17 @@ struct MlpParams {
   int row_cap;
 };
 
+// A contiguous sub-batch of chains [start, start + n) with its own bookkeeping.  The whole batch is one
+// lane; asd_sample may split it into two that take turns (see asd_api.cu).
+struct Lane {
+  int start = 0, n = 0;
+  int* act = nullptr;        // [n] active position -> chain position inside the lane
+  int* row_off = nullptr;    // [n + 1]
+  int* step1 = nullptr;      // [n]
+  RoundCounters* counters = nullptr;
+  int* v_off = nullptr;      // device int: row of the drift buffer where this lane's v_a rows start
+};
+
 // Phases of a round, for the optional per-phase CUDA-event timing.
 enum Phase {
   PH_PREP = 0, PH_PACK, PH_D1_IN, PH_D1_HID, PH_D1_OUT, PH_D1_ANALYTIC, PH_DRAFT,
@@ -173,9 +184,15 @@ void prof_collect_some(Ctx* c, long long count);
 void prof_collect(Ctx* c);  // after a stream synchronisation: fold pending event pairs into c->prof
 
 // ---- launchers (asd_kernels.cu) ---------------------------------------------------------
-void launch_prep(Ctx* c, int window);
-void launch_draft(Ctx* c, int window);
-void launch_verify(Ctx* c, int window, bool use_u);
+Lane whole_batch(const Ctx* c);
+void launch_prep(Ctx* c, const Lane& L, int window);
+// v_base + (*v_off_dev) rows: where the lane's v_a rows are (v_off_dev may be null: offset 0)
+void launch_draft(Ctx* c, const Lane& L, int window, const float* v_base, const int* v_off_dev);
+void launch_verify(Ctx* c, const Lane& L, int window, bool use_u, const float* G, const float* v_base,
+                   const int* v_off_dev);
+// Pass-1 rows of lane L appended behind the drafted rows of the other lane: row = *row_base_dev + p gets
+// the point y_a, its network input, step and slot; *m_merged_dev = *row_base_dev + active chains of L.
+void launch_pack_appended(Ctx* c, const Lane& L, const int* row_base_dev, int* m_merged_dev);
 void launch_pack(Ctx* c, const RowSet& rs);
 void launch_gmm(Ctx* c, const RowSet& rs, float* out);
 void launch_gauss(Ctx* c, const RowSet& rs, float* out);

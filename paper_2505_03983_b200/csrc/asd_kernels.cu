@@ -4,6 +4,8 @@
 // of the network denoiser.  fp32 throughout; the Gaussian noise uses the special-function unit's
 // approximate lg2 / sqrt / sin / cos (absolute error about 1e-6 per normal), everything that decides an
 // accept test (ln u, the reductions) is plain IEEE fp32.
+#include <algorithm>
+
 #include "asd_internal.h"
 
 namespace asd {
@@ -196,9 +198,21 @@ __global__ void __launch_bounds__(1024) prep_kernel(const int* __restrict__ a, c
 // Per-chain speculation lengths apply to speculation rounds only (never to the window-1 steps of Eq. 7).
 static const int* round_windows(const Ctx* c, int window) { return (c->adaptive && window > 1) ? c->wnd : nullptr; }
 
-void launch_prep(Ctx* c, int window) {
-  prep_kernel<<<1, 1024, 0, c->stream>>>(c->a, round_windows(c, window), c->n, c->K, window, c->act, c->row_off, c->step1, c->acc_len,
-                                         c->counters);
+Lane whole_batch(const Ctx* c) {
+  Lane L;
+  L.start = 0;
+  L.n = c->n;
+  L.act = c->act;
+  L.row_off = c->row_off;
+  L.step1 = c->step1;
+  L.counters = c->counters;
+  return L;
+}
+
+void launch_prep(Ctx* c, const Lane& L, int window) {
+  const int* wnd = round_windows(c, window);
+  prep_kernel<<<1, 1024, 0, c->stream>>>(c->a + L.start, wnd ? wnd + L.start : nullptr, L.n, c->K, window, L.act, L.row_off,
+                                         L.step1, c->acc_len + L.start, L.counters);
   c->launches++;
 }
 
@@ -223,6 +237,7 @@ struct DraftArgs {
   const int* row_off;
   const float* y;
   const float* v;
+  const int* v_off;  // device: first row of v for this lane, or null
   Tables tab;
   float* Yhat;
   int* row_step;
@@ -274,7 +289,7 @@ __global__ void __launch_bounds__(kDraftThreads) draft_kernel(const DraftArgs A)
     const int q = blockIdx.x * kDraftThreads + threadIdx.x;
     if (q < A.nq) {
       float4 yh = load4(A.y + (size_t)j * A.d, q, A.d, A.vec);
-      const float4 v = load4(A.v + (size_t)p * A.d, q, A.d, A.vec);
+      const float4 v = load4(A.v + (size_t)((A.v_off ? *A.v_off : 0) + p) * A.d, q, A.d, A.vec);
       for (int k = 1; k < w; ++k) {
         const int i = a + k - 1;  // step i -> i+1 uses eta_i, sigma_{i+1}, xi_{i+1}
         const float eta = A.tab.eta[i], sig = A.tab.sig[i];
@@ -297,7 +312,7 @@ __global__ void __launch_bounds__(kDraftThreads) draft_kernel(const DraftArgs A)
     __syncthreads();
     if (ks == 0 && q_ok) {
       float4 yh = load4(A.y + (size_t)j * A.d, q, A.d, A.vec);
-      const float4 v = load4(A.v + (size_t)p * A.d, q, A.d, A.vec);
+      const float4 v = load4(A.v + (size_t)((A.v_off ? *A.v_off : 0) + p) * A.d, q, A.d, A.vec);
       for (int k = 1; k < w; ++k) {
         const int i = a + k - 1;
         const float eta = A.tab.eta[i], sig = A.tab.sig[i];
@@ -335,8 +350,9 @@ __global__ void __launch_bounds__(kDraftThreads) draft_kernel(const DraftArgs A)
   }
 }
 
-void launch_draft(Ctx* c, int window) {
-  if (window <= 1 || c->n == 0) return;
+void launch_draft(Ctx* c, const Lane& L, int window, const float* v_base, const int* v_off_dev) {
+  if (window <= 1 || L.n == 0) return;
+  const int* wnd = round_windows(c, window);
   DraftArgs A{};
   A.d = c->d;
   A.K = c->K;
@@ -344,14 +360,15 @@ void launch_draft(Ctx* c, int window) {
   A.nq = (c->d + 3) / 4;
   A.vec = (c->d % 4 == 0);
   A.keys = make_philox_keys(c->seed);
-  A.chain_base = c->chain_base;
-  A.cnt = c->counters;
-  A.act = c->act;
-  A.a = c->a;
-  A.wnd = round_windows(c, window);
-  A.row_off = c->row_off;
-  A.y = c->y;
-  A.v = c->v;
+  A.chain_base = c->chain_base + (uint64_t)L.start;
+  A.cnt = L.counters;
+  A.act = L.act;
+  A.a = c->a + L.start;
+  A.wnd = wnd ? wnd + L.start : nullptr;
+  A.row_off = L.row_off;
+  A.y = c->y + (size_t)L.start * c->d;
+  A.v = v_base;
+  A.v_off = v_off_dev;
   A.tab = c->tab;
   A.Yhat = c->Yhat;
   A.row_step = c->row_step;
@@ -362,13 +379,13 @@ void launch_draft(Ctx* c, int window) {
     A.in_dim = c->mlp.in_dim;
     A.d_cond = c->mlp.d_cond;
     A.d_temb = c->mlp.d_temb;
-    A.cond = c->mlp.cond;
+    A.cond = c->mlp.cond + (size_t)L.start * c->mlp.d_cond;
     A.temb = c->mlp.temb;
   }
   // the staged, slot-parallel form only when one thread per 4 dims would leave the machine mostly idle
-  A.par = (long long)c->n * ((A.nq + kDraftThreads - 1) / kDraftThreads) < 2ll * c->num_sms;
+  A.par = (long long)L.n * ((A.nq + kDraftThreads - 1) / kDraftThreads) < 2ll * c->num_sms;
   const int per_block = A.par ? kDraftQ : kDraftThreads;
-  dim3 grid((A.nq + per_block - 1) / per_block, c->n);
+  dim3 grid((A.nq + per_block - 1) / per_block, L.n);
   draft_kernel<<<grid, kDraftThreads, 0, c->stream>>>(A);
   c->launches++;
 }
@@ -402,6 +419,7 @@ struct VerifyArgs {
   const int* row_off;
   float* y;
   const float* v;
+  const int* v_off;  // device: first row of v for this lane, or null
   const float* Yhat;
   const float* G;
   Tables tab;
@@ -423,7 +441,7 @@ __global__ void __launch_bounds__(256) verify_kernel(const VerifyArgs A) {
   const int row0 = A.row_off[p];
   const uint32_t chain = (uint32_t)(A.chain_base + (uint64_t)j);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
-  const float* vrow = A.v + (size_t)p * A.d;
+  const float* vrow = A.v + (size_t)((A.v_off ? *A.v_off : 0) + p) * A.d;
   const float nan = __int_as_float(0x7fc00000);
 
   // ln u of every slot (one Philox call each), and the diagnostics of slot 1: proposal mean == target
@@ -570,8 +588,10 @@ __global__ void __launch_bounds__(256) verify_kernel(const VerifyArgs A) {
   }
 }
 
-void launch_verify(Ctx* c, int window, bool use_u) {
-  if (c->n == 0) return;
+void launch_verify(Ctx* c, const Lane& L, int window, bool use_u, const float* G, const float* v_base,
+                   const int* v_off_dev) {
+  if (L.n == 0) return;
+  const int* wnd = round_windows(c, window);
   VerifyArgs A{};
   A.d = c->d;
   A.K = c->K;
@@ -581,26 +601,27 @@ void launch_verify(Ctx* c, int window, bool use_u) {
   A.use_u = use_u;
   A.all_slots = c->debug_all_slots ? 1 : 0;
   A.dbg_stride = c->window;
-  A.wnd = const_cast<int*>(round_windows(c, window));
-  A.ema8 = c->ema8;
+  A.wnd = wnd ? const_cast<int*>(wnd) + L.start : nullptr;
+  A.ema8 = c->ema8 + L.start;
   A.keys = make_philox_keys(c->seed);
-  A.chain_base = c->chain_base;
-  A.cnt = c->counters;
-  A.act = c->act;
-  A.a = c->a;
-  A.rounds = c->rounds;
-  A.row_off = c->row_off;
-  A.y = c->y;
-  A.v = c->v;
+  A.chain_base = c->chain_base + (uint64_t)L.start;
+  A.cnt = L.counters;
+  A.act = L.act;
+  A.a = c->a + L.start;
+  A.rounds = c->rounds + L.start;
+  A.row_off = L.row_off;
+  A.y = c->y + (size_t)L.start * c->d;
+  A.v = v_base;
+  A.v_off = v_off_dev;
   A.Yhat = c->Yhat;
-  A.G = c->G;
+  A.G = G;
   A.tab = c->tab;
-  A.dbg_lr = c->dbg_lr;
-  A.dbg_lu = c->dbg_lu;
-  A.acc_len = c->acc_len;
+  A.dbg_lr = c->dbg_lr + (size_t)L.start * c->window;
+  A.dbg_lu = c->dbg_lu + (size_t)L.start * c->window;
+  A.acc_len = c->acc_len + L.start;
   // eight warps per chain; a slot is reduced by two warps when a row has >= 512 float4 groups, else by one
   A.wps = A.nq >= 512 ? 2 : 1;
-  verify_kernel<<<c->n, 256, 0, c->stream>>>(A);
+  verify_kernel<<<L.n, 256, 0, c->stream>>>(A);
   c->launches++;
 }
 
@@ -710,6 +731,58 @@ void launch_pack(Ctx* c, const RowSet& rs) {
   if (rs.n_rows_max <= 0) return;
   int blocks = rs.n_rows_max > 8 * c->num_sms ? 8 * c->num_sms : rs.n_rows_max;
   pack_kernel<<<blocks, 256, 0, c->stream>>>(rs, c->d, c->mlp, c->tab.c_in);
+  c->launches++;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Pass-1 rows of one lane appended behind the drafted rows of the other (staggered lanes): the point y_a
+// of active chain p becomes row *row_base + p of the drafted-point buffer, with its network input row,
+// step and slot, so that one GEMM pass serves both lanes.
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) pack_appended_kernel(const RoundCounters* __restrict__ cnt, const int* __restrict__ act,
+                                                            const int* __restrict__ a, const float* __restrict__ y,
+                                                            const int* __restrict__ row_base, int* __restrict__ m_merged,
+                                                            int* __restrict__ v_off, int d, MlpParams M,
+                                                            const __nv_bfloat16* __restrict__ cond,
+                                                            const float* __restrict__ c_in, float* __restrict__ Yhat,
+                                                            int* __restrict__ row_step, int* __restrict__ row_slot) {
+  const int n_active = cnt->n_active, base = *row_base;
+  if (blockIdx.x == 0 && threadIdx.x == 0) {
+    *m_merged = base + n_active;
+    *v_off = base;
+  }
+  for (int p = blockIdx.x; p < n_active; p += gridDim.x) {
+    const int j = act[p], step = a[j], row = base + p;
+    const float* yj = y + (size_t)j * d;
+    const float ci = c_in[step];
+    float* yr = Yhat + (size_t)row * d;
+    __nv_bfloat16* xr = M.X + (size_t)row * M.in_pad;
+    for (int e = threadIdx.x; e < M.in_pad; e += blockDim.x) {
+      __nv_bfloat16 val = __float2bfloat16_rn(0.f);
+      if (e < d) {
+        const float yv = yj[e];
+        yr[e] = yv;
+        val = __float2bfloat16_rn(ci * yv);
+      } else if (e < d + M.d_cond) {
+        val = cond[(size_t)j * M.d_cond + (e - d)];
+      } else if (e < M.in_dim) {
+        val = M.temb[(size_t)step * M.d_temb + (e - d - M.d_cond)];
+      }
+      xr[e] = val;
+    }
+    if (threadIdx.x == 0) {
+      row_step[row] = step;
+      row_slot[row] = j;
+    }
+  }
+}
+
+void launch_pack_appended(Ctx* c, const Lane& L, const int* row_base_dev, int* m_merged_dev) {
+  int blocks = std::max(1, std::min(L.n, 8 * c->num_sms));
+  pack_appended_kernel<<<blocks, 256, 0, c->stream>>>(L.counters, L.act, c->a + L.start, c->y + (size_t)L.start * c->d,
+                                                      row_base_dev, m_merged_dev, L.v_off, c->d, c->mlp,
+                                                      c->mlp.cond + (size_t)L.start * c->mlp.d_cond, c->tab.c_in, c->Yhat,
+                                                      c->row_step, c->row_slot);
   c->launches++;
 }
 
