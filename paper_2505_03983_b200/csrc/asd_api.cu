@@ -138,15 +138,13 @@ int bound_bucket(const Ctx* c, int active) {
 
 // Enqueues one round on c->stream (which must be the context's private stream): replays the captured
 // graph for this shape, capturing it on first use.
-asd_status launch_round_graph(Ctx* c, int window, bool use_u, int active) {
-  if (active <= 0) return ASD_OK;
-  const int bucket = bound_bucket(c, active);
-  const auto key = std::make_tuple(window, use_u ? 1 : 0, bucket);
+template <typename Body>
+asd_status launch_captured(Ctx* c, const std::tuple<int, int, long long>& key, Body body) {
   auto it = c->graphs.find(key);
   if (it == c->graphs.end()) {
     const long long l0 = c->launches;
     ASD_CUDA(c, cudaStreamBeginCapture(c->stream, cudaStreamCaptureModeThreadLocal));
-    const asd_status st = enqueue_round(c, window, use_u, bucket);
+    const asd_status st = body();
     cudaGraph_t graph = nullptr;
     const cudaError_t e = cudaStreamEndCapture(c->stream, &graph);
     const long long captured = c->launches - l0;
@@ -165,6 +163,65 @@ asd_status launch_round_graph(Ctx* c, int window, bool use_u, int active) {
   ASD_CUDA(c, cudaGraphLaunch(it->second.exec, c->stream));
   c->launches += it->second.launches;
   return ASD_OK;
+}
+
+asd_status launch_round_graph(Ctx* c, int window, bool use_u, int active) {
+  if (active <= 0) return ASD_OK;
+  const int bucket = bound_bucket(c, active);
+  return launch_captured(c, std::make_tuple(window, use_u ? 1 : 0, (long long)bucket),
+                         [&] { return enqueue_round(c, window, use_u, bucket); });
+}
+
+// One tick of the staggered schedule (network denoiser).  The batch is split into two lanes that run
+// Algorithm 1's round half a round apart: in tick t lane Y = t mod 2 is at its first model call (drift
+// at the current points) and lane X = the other one at its second (drift at its drafted points), and both
+// go through ONE pass of the GEMM chain: Y's current points are appended as rows behind X's drafted
+// rows.  Then X is verified and advanced, and Y drafts its window from the drifts it just received.  Per
+// chain nothing changes (same rounds, same arithmetic); the pass with very few rows disappears.
+// The drift buffer alternates between ticks because X's v_a rows, produced a tick earlier, are still
+// needed by its verify step.
+asd_status enqueue_tick(Ctx* c, long long t, int window, int bound_x, int bound_y) {
+  Lane& Y = c->lanes[t & 1];
+  Lane& X = c->lanes[(t + 1) & 1];
+  float* g_cur = (t & 1) ? c->G2 : c->G;
+  const float* g_prev = (t & 1) ? c->G : c->G2;
+  {
+    ProfScope ps(c, PH_PREP);
+    launch_prep(c, Y, window);
+  }
+  {
+    ProfScope ps(c, PH_PACK);
+    launch_pack_appended(c, Y, &X.counters->rows2, c->merged_rows);
+  }
+  RowSet rs{c->merged_rows, bound_x * (window - 1) + bound_y, c->Yhat, nullptr, c->row_step, c->row_slot};
+  asd_status st = mlp_forward(c, rs, g_cur, 1);
+  if (st != ASD_OK) return st;
+  {
+    ProfScope ps(c, PH_VERIFY);
+    launch_verify(c, X, window, true, g_cur, g_prev, X.v_off);
+  }
+  {
+    ProfScope ps(c, PH_DRAFT);
+    launch_draft(c, Y, window, g_cur, Y.v_off);
+  }
+  ASD_CUDA(c, cudaGetLastError());
+  return ASD_OK;
+}
+
+int lane_bucket(int active, int n) {
+  if (active >= n) return n;
+  int b = 1;
+  while (b < active) b <<= 1;
+  return std::min(b, n);
+}
+
+asd_status launch_tick(Ctx* c, bool graphs, long long t, int window, int act_x, int act_y) {
+  const Lane& Y = c->lanes[t & 1];
+  const Lane& X = c->lanes[(t + 1) & 1];
+  const int bx = lane_bucket(act_x, X.n), by = lane_bucket(act_y, Y.n);
+  if (!graphs) return enqueue_tick(c, t, window, bx, by);
+  return launch_captured(c, std::make_tuple(window, 2 + (int)(t & 1), (long long)bx * (1ll << 32) + by),
+                         [&] { return enqueue_tick(c, t, window, bx, by); });
 }
 
 // While alive, the context's work goes to its private stream, ordered after what the caller's stream
@@ -190,6 +247,89 @@ struct PrivateStreamScope {
 
 asd_status enqueue_round_any(Ctx* c, bool graphs, int window, bool use_u, int active) {
   return graphs ? launch_round_graph(c, window, use_u, active) : enqueue_round(c, window, use_u, active);
+}
+
+// Whether asd_sample runs the batch as two staggered lanes (network denoiser only).  Off unless
+// ASD_STAGGER=1: measured on B200 it does not pay - at 512 x 64 and 2048 x 64 chains x window the pass with
+// few rows that it removes (6 % and 3 % of the step) is offset by the less efficient half-size GEMM launches
+// and the doubled draft / verify launches (936 against 920 ms and 3583 against 3545 ms per step); the
+// run is bound by the power cap, so what counts is energy per FLOP, not idle gaps.
+bool use_stagger(const Ctx* c) {
+  if (c->kind != ASD_DEN_RESMLP_BF16 || !c->G2 || c->window < 4 || c->n < 2) return false;
+  const char* e = getenv("ASD_STAGGER");
+  return e && e[0] == '1';
+}
+
+// asd_sample for two staggered lanes: same run-ahead scheme as below, one ring slot per tick holding both
+// lanes' counters and the merged row count.
+asd_status sample_staggered(Ctx* c) {
+  constexpr int kDepth = 4;
+  constexpr size_t kEventsPerTick = 2 * PH_COUNT + 8;
+  int active[2] = {c->lanes[0].n, c->lanes[1].n};
+  long long issued = 0, consumed = 0;
+  const long long max_ticks = 2ll * c->K + 6;
+  size_t prof_pairs[Ctx::kRing] = {};
+  asd_status deferred = ASD_OK;
+  PrivateStreamScope pss(c);
+  auto consume = [&](bool wait) -> bool {
+    const int slot = (int)(consumed % Ctx::kRing);
+    if (wait) {
+      if (cudaEventSynchronize(c->ring_ev[slot]) != cudaSuccess) {
+        deferred = fail(c, ASD_ERR_CUDA, "event synchronisation failed");
+        return false;
+      }
+    } else if (cudaEventQuery(c->ring_ev[slot]) != cudaSuccess) {
+      return false;
+    }
+    const long long t = consumed;
+    const RoundCounters& hy = c->ring_host[3 * slot + (t & 1)];        // lane at its first model call
+    const RoundCounters& hx = c->ring_host[3 * slot + ((t + 1) & 1)];  // lane that was verified
+    const int merged = c->ring_host[3 * slot + 2].n_active;
+    if (t >= 1) active[(t + 1) & 1] = hx.n_active_after;  // tick 0 verifies nothing
+    if (c->prof_on) {
+      prof_collect_some(c, (long long)prof_pairs[slot]);
+      for (int ph : {PH_PREP, PH_PACK, PH_DRAFT}) c->prof[ph].rows += hy.n_active;
+      c->prof[PH_VERIFY].rows += hx.n_active;
+      for (int ph : {PH_D2_IN, PH_D2_HID, PH_D2_OUT}) c->prof[ph].rows += merged;
+    }
+    ++consumed;
+    return true;
+  };
+  while ((active[0] > 0 || active[1] > 0) && issued < max_ticks && deferred == ASD_OK) {
+    const long long t = issued;
+    const int slot = (int)(t % Ctx::kRing);
+    c->ev_used = (size_t)slot * kEventsPerTick;
+    const size_t pending0 = c->pending.size();
+    asd_status st = launch_tick(c, pss.on, t, c->window, active[(t + 1) & 1], active[t & 1]);
+    if (st != ASD_OK) return st;
+    prof_pairs[slot] = c->pending.size() - pending0;
+    for (int l = 0; l < 2; ++l)
+      ASD_CUDA(c, cudaMemcpyAsync(&c->ring_host[3 * slot + l], c->lanes[l].counters, sizeof(RoundCounters),
+                                  cudaMemcpyDeviceToHost, c->stream));
+    ASD_CUDA(c, cudaMemcpyAsync(&c->ring_host[3 * slot + 2].n_active, c->merged_rows, sizeof(int), cudaMemcpyDeviceToHost,
+                                c->stream));
+    ASD_CUDA(c, cudaEventRecord(c->ring_ev[slot], c->stream));
+    ++issued;
+    while (consumed < issued && consume(issued - consumed >= kDepth)) {
+    }
+  }
+  while (consumed < issued && deferred == ASD_OK && consume(true)) {
+  }
+  if (deferred != ASD_OK) {
+    cudaStreamSynchronize(c->stream);
+    prof_collect(c);
+    return deferred;
+  }
+  if (active[0] > 0 || active[1] > 0) return fail(c, ASD_ERR_STATE, "chains still active after 2K ticks");
+  // the lanes' running totals (the last ring slot holds their final counters)
+  if (issued > 0) {
+    const int slot = (int)((issued - 1) % Ctx::kRing);
+    for (int l = 0; l < 2; ++l) {
+      c->extra_rows_total += (long long)c->ring_host[3 * slot + l].rows_total;
+      c->extra_rows_verified += (long long)c->ring_host[3 * slot + l].rows_verified;
+    }
+  }
+  return ASD_OK;
 }
 
 }  // namespace
@@ -374,9 +514,9 @@ asd_status asd_create(const asd_config* cfg, void* cuda_stream, asd_ctx** out) {
         cudaEventCreateWithFlags(&c->join_ev, cudaEventDisableTiming) != cudaSuccess)
       return abandon(fail(c, ASD_ERR_CUDA, "stream / event creation failed"));
   }
-  if (cudaMallocHost(&c->ring_host, Ctx::kRing * sizeof(RoundCounters)) != cudaSuccess)
+  if (cudaMallocHost(&c->ring_host, 3 * Ctx::kRing * sizeof(RoundCounters)) != cudaSuccess)
     return abandon(fail(c, ASD_ERR_OOM, "pinned allocation failed"));
-  memset(c->ring_host, 0, Ctx::kRing * sizeof(RoundCounters));
+  memset(c->ring_host, 0, 3 * Ctx::kRing * sizeof(RoundCounters));
   for (int i = 0; i < Ctx::kRing; ++i)
     if (cudaEventCreateWithFlags(&c->ring_ev[i], cudaEventDisableTiming) != cudaSuccess)
       return abandon(fail(c, ASD_ERR_CUDA, "event creation failed"));
@@ -507,6 +647,15 @@ asd_status asd_create(const asd_config* cfg, void* cuda_stream, asd_ctx** out) {
     TRY(dev_alloc(c, &M.X, (size_t)M.row_cap * M.in_pad));
     TRY(dev_alloc(c, &M.H[0], (size_t)M.row_cap * W));
     TRY(dev_alloc(c, &M.H[1], (size_t)M.row_cap * W));
+    TRY(dev_alloc(c, &c->G2, R * d));
+    TRY(dev_alloc(c, &c->merged_rows, 4));
+    for (int l = 0; l < 2; ++l) {
+      TRY(dev_alloc(c, &c->lanes[l].act, n));
+      TRY(dev_alloc(c, &c->lanes[l].row_off, n + 1));
+      TRY(dev_alloc(c, &c->lanes[l].step1, n));
+      TRY(dev_alloc(c, &c->lanes[l].counters, 1));
+      TRY(dev_alloc(c, &c->lanes[l].v_off, 4));
+    }
   }
 #undef TRY
   if (cudaStreamSynchronize(c->stream) != cudaSuccess) return abandon(fail(c, ASD_ERR_CUDA, "create: sync failed"));
@@ -539,6 +688,18 @@ asd_status asd_reset(asd_ctx* ctx, int32_t n_chains, uint64_t chain_id_base, con
   ASD_CUDA(c, cudaMemsetAsync(c->rounds, 0, (size_t)c->max_chains * sizeof(int), c->stream));
   ASD_CUDA(c, cudaMemsetAsync(c->counters, 0, 2 * sizeof(RoundCounters), c->stream));
   launch_fill_int(c, c->acc_len, c->max_chains, -1);
+  if (c->G2) {
+    const int h = (n_chains + 1) / 2;
+    c->lanes[0].start = 0;
+    c->lanes[0].n = h;
+    c->lanes[1].start = h;
+    c->lanes[1].n = n_chains - h;
+    for (int l = 0; l < 2; ++l) {
+      ASD_CUDA(c, cudaMemsetAsync(c->lanes[l].counters, 0, sizeof(RoundCounters), c->stream));
+      ASD_CUDA(c, cudaMemsetAsync(c->lanes[l].v_off, 0, sizeof(int), c->stream));
+    }
+    ASD_CUDA(c, cudaMemsetAsync(c->merged_rows, 0, sizeof(int), c->stream));
+  }
   // adaptive mode starts every chain at 8 x mean = 32, i.e. a speculation length of min(window, 8)
   launch_fill_int(c, c->ema8, c->max_chains, kAdaptInitEma8);
   launch_fill_int(c, c->wnd, c->max_chains, std::max(2, std::min(c->window, 2 + (3 * kAdaptInitEma8) / 16)));
@@ -585,8 +746,8 @@ static asd_status finish_run(Ctx* c, float* y_out_dev, int32_t* rounds_out_dev, 
     float ms = 0.f;
     cudaEventElapsedTime(&ms, c->ev0, c->ev1);
     stats->ms_total = ms;
-    stats->rows_total = (int64_t)c->counters_host->rows_total;
-    stats->rows_verified = (int64_t)c->counters_host->rows_verified;
+    stats->rows_total = (int64_t)c->counters_host->rows_total + c->extra_rows_total;
+    stats->rows_verified = (int64_t)c->counters_host->rows_verified + c->extra_rows_verified;
     stats->launches = c->launches - launches0;
     stats->rounds_max = 0;
     stats->rounds_mean = 0.0;
@@ -617,6 +778,12 @@ asd_status asd_sample(asd_ctx* ctx, float* y_out_dev, int32_t* rounds_out_dev, a
   // bound on the active chains that sizes the grids is therefore a few rounds old, which is still an
   // upper bound (chains only finish), and the rounds enqueued after the last chain finished find no
   // active chain and do nothing.  Theorem 3: the cursor strictly increases, so K rounds always suffice.
+  c->extra_rows_total = c->extra_rows_verified = 0;
+  if (use_stagger(c)) {
+    asd_status st = sample_staggered(c);
+    if (st != ASD_OK) return st;
+    return finish_run(c, y_out_dev, rounds_out_dev, stats_host, launches0, true);
+  }
   // Unless per-phase timing is on, a round is replayed as one CUDA graph on the context's private stream.
   constexpr int kDepth = 4;
   int active = c->n;

@@ -1048,10 +1048,8 @@ asd_status launch_gemm_skinny(Ctx* c, const void* a_ptr, int a_cols, const void*
 
 // Few rows: weight streaming with swapped operands.  (ASD_GEMM_MODE=cta|pair pins the tiled kernels.)
 bool use_skinny(int m_bound) {
-  static const bool pinned = [] {
-    const char* e = getenv("ASD_GEMM_MODE");
-    return e && (!strcmp(e, "cta") || !strcmp(e, "pair"));
-  }();
+  const char* e = getenv("ASD_GEMM_MODE");
+  const bool pinned = e && (!strcmp(e, "cta") || !strcmp(e, "pair"));
   return !pinned && m_bound <= kSkinnyMaxRows;
 }
 
@@ -1064,10 +1062,8 @@ struct GemmPlan {
 };
 
 GemmPlan plan_gemm(const Ctx* c, int m_bound, int n_out) {
-  static const int mode = [] {
-    const char* e = getenv("ASD_GEMM_MODE");  // tuning aid: "cta" or "pair" pins the kernel family
-    return !e ? 0 : (!strcmp(e, "cta") ? 1 : (!strcmp(e, "pair") ? 2 : 0));
-  }();
+  const char* e = getenv("ASD_GEMM_MODE");  // tuning aid: "cta" or "pair" pins the kernel family
+  const int mode = !e ? 0 : (!strcmp(e, "cta") ? 1 : (!strcmp(e, "pair") ? 2 : 0));
   const double fill_rate = 50.0;
   GemmPlan best{false, 32};
   double best_t = 1e300;

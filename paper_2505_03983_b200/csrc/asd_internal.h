@@ -135,6 +135,12 @@ struct Ctx {
   float* v = nullptr;        // [max_chains, d] drift at the current point, by active position
   float* Yhat = nullptr;     // [max_rows, d] drafted points y^_{a+k}, k = 1..w-1
   float* G = nullptr;        // [max_rows, d] drift at the drafted points
+  // staggered lanes (network denoiser): second drift buffer (ticks alternate), the two half-batches, the
+  // row count of a merged pass
+  float* G2 = nullptr;
+  Lane lanes[2];
+  int* merged_rows = nullptr;
+  long long extra_rows_total = 0, extra_rows_verified = 0;  // lanes' counters, added by the run statistics
   float* dbg_lr = nullptr;   // [max_chains, window]
   float* dbg_lu = nullptr;   // [max_chains, window]
   int* acc_len = nullptr;    // [max_chains]
@@ -143,7 +149,7 @@ struct Ctx {
   // asd_sample runs ahead of the device: the counters of round r land in ring_host[r % kRing] and
   // ring_ev[r % kRing] tells when
   static constexpr int kRing = 8;
-  RoundCounters* ring_host = nullptr;      // pinned [kRing]
+  RoundCounters* ring_host = nullptr;      // pinned [kRing][3]: whole batch or lane 0, lane 1, merged row count
   cudaEvent_t ring_ev[kRing] = {};
   int max_rows = 0;
   Tables tab{};
@@ -155,7 +161,7 @@ struct Ctx {
   // One speculation round captured as a CUDA graph per (window, use_u, bound on active chains); replayed
   // on a private stream that is forked from and joined to the caller's stream.
   struct RoundGraph { cudaGraphExec_t exec; long long launches; };
-  std::map<std::tuple<int, int, int>, RoundGraph> graphs;
+  std::map<std::tuple<int, int, long long>, RoundGraph> graphs;
   cudaStream_t gstream = nullptr;
   cudaEvent_t fork_ev = nullptr, join_ev = nullptr;
   bool use_graphs = true;
