@@ -109,6 +109,13 @@ def oracle_sample_rate(wl, budget_s: float, max_rounds: int):
     return frac / el, f"chain 0, first {rounds} rounds ({a} of {wl.K} steps) in {el:.1f} s, extrapolated by steps"
 
 
+def config_of(wl):
+    return {"workload": wl.name, "chains_per_gpu": wl.chains, "K": wl.K, "window": wl.window, "d": wl.d,
+            "denoiser": wl.kind, "width": wl.width, "layers": wl.n_layers,
+            "l2": "working set (weights + activations) larger than L2, no flush needed"
+                  if wl.kind == "mlp" and wl.width >= 4096 else "small working set; L2-resident by design"}
+
+
 def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
@@ -132,7 +139,7 @@ def run_reference(args):
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * el / max(args.steps, 1),
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": wl.name, "chains": wl.chains, "K": wl.K, "window": wl.window, "d": wl.d},
+        "config": config_of(wl),
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
                          "sample": "each step: " + desc},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -265,10 +272,7 @@ def run_ours(args):
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16" if wl.kind == "mlp" else "f32", "data": "synthetic",
-        "config": {"workload": wl.name, "chains_per_gpu": n, "K": wl.K, "window": wl.window, "d": wl.d,
-                   "denoiser": wl.kind, "width": wl.width, "layers": wl.n_layers,
-                   "l2": "working set (weights + activations) larger than L2, no flush needed"
-                         if wl.kind == "mlp" and wl.width >= 4096 else "small working set; L2-resident by design"},
+        "config": config_of(wl),
         "rounds_per_sample": float(np.mean(rounds_mean)), "rounds_max": int(max(rounds_max)),
         "K_over_rounds": wl.K / float(np.mean(rounds_mean)),
         "drift_rows_per_sample_over_K": rows / (args.steps * n * wl.K),
