@@ -384,6 +384,30 @@ def test_empty_and_degenerate_inputs():
         _sampler(bad)
 
 
+def test_degenerate_constant_drift_accepts_everything():
+    """A drift that does not depend on the point (zero output weights, no skip) makes proposal and target
+    means equal at every slot: ratio exactly 1, |delta|^2 = 0, every window accepted whole, so each chain
+    needs exactly ceil(K / window) rounds and ends where the sequential sampler ends, bit for bit."""
+    wl = workloads.make("mlp_tiny", K=37, window=6, chains=5)
+    wl.W_out[:] = 0
+    wl.c_skip[:] = 0
+    wl.c_out[:] = 0.5                 # g = 0.5 b_out at every step and point
+    with _sampler(wl) as s:
+        s.reset(5, 3, cond=wl.cond)
+        y, r, st = s.sample()
+        s.reset(5, 3, cond=wl.cond)
+        st1 = s.round()
+        lr, lu, acc = s.debug_last_round()
+        s.reset(5, 3, cond=wl.cond)
+        y_seq, _ = s.sequential_ddpm()
+    assert torch.all(r == math.ceil(37 / 6)) and st.rows_total == 5 * (6 * 6 + 1)
+    assert torch.all(acc == 6) and st1.accepted_total == 30 and torch.all(lr == 0)
+    assert torch.equal(y, y_seq)
+    g, sch = oden.from_workload(wl), oasd.make_schedule(wl.t)
+    res = oasd.asd_sample(g, sch, wl.seed, 3, 0, 6, d=wl.d)
+    assert res.rounds == 7 and rel_l2(y[0].cpu().numpy().astype(np.float64), res.y) < 1e-5
+
+
 def test_gaussian_target_moments_many_chains():
     """cfg-2 statistical check on the GPU: 16384 ASD chains and 16384 sequential chains against the
     closed-form law of the Euler chain (mean T mu0, eigen-variances (1+T lam)^2 sum eta/(1+t lam)^2)."""
