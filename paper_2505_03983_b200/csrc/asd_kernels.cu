@@ -277,7 +277,7 @@ __device__ __forceinline__ void draft_store(const DraftArgs& A, int row, int a, 
 
 __global__ void __launch_bounds__(kDraftThreads) draft_kernel(const DraftArgs A) {
   __shared__ float4 s_pt[kMaxWindow - 1][kDraftQ];  // noise, then drafted points, per slot (parallel form)
-  const int p = blockIdx.y;
+  const int p = blockIdx.x;
   if (p >= A.cnt->n_active) return;
   const int j = A.act[p];
   const int a = A.a[j];
@@ -286,7 +286,7 @@ __global__ void __launch_bounds__(kDraftThreads) draft_kernel(const DraftArgs A)
   const uint32_t chain = (uint32_t)(A.chain_base + (uint64_t)j);
   if (!A.par) {
     // large batches: one thread owns 4 dims and walks the window; nothing is staged
-    const int q = blockIdx.x * kDraftThreads + threadIdx.x;
+    const int q = blockIdx.y * kDraftThreads + threadIdx.x;
     if (q < A.nq) {
       float4 yh = load4(A.y + (size_t)j * A.d, q, A.d, A.vec);
       const float4 v = load4(A.v + (size_t)((A.v_off ? *A.v_off : 0) + p) * A.d, q, A.d, A.vec);
@@ -305,7 +305,7 @@ __global__ void __launch_bounds__(kDraftThreads) draft_kernel(const DraftArgs A)
     // small batches: the noise of all slots in parallel, then the recurrence by one warp, then the stores
     const int ql = threadIdx.x & (kDraftQ - 1), ks = threadIdx.x / kDraftQ;
     constexpr int kSlotLanes = kDraftThreads / kDraftQ;
-    const int q = blockIdx.x * kDraftQ + ql;
+    const int q = blockIdx.y * kDraftQ + ql;
     const bool q_ok = q < A.nq;
     if (q_ok)
       for (int k = 1 + ks; k < w; k += kSlotLanes) s_pt[k - 1][ql] = xi4((uint32_t)q, (uint32_t)(a + k), chain, A.keys);
@@ -329,7 +329,7 @@ __global__ void __launch_bounds__(kDraftThreads) draft_kernel(const DraftArgs A)
       for (int k = 1 + ks; k < w; k += kSlotLanes) draft_store(A, row0 + k - 1, a, k, q, s_pt[k - 1][ql]);
   }
   // row maps, conditioning, time embedding and zero padding: the chain's blocks share the slots
-  for (int k = 1 + (int)blockIdx.x; k < w; k += gridDim.x) {
+  for (int k = 1 + (int)blockIdx.y; k < w; k += gridDim.y) {
     const int row = row0 + k - 1;
     if (threadIdx.x == 0) {
       A.row_step[row] = a + k;
@@ -385,7 +385,7 @@ void launch_draft(Ctx* c, const Lane& L, int window, const float* v_base, const 
   // the staged, slot-parallel form only when one thread per 4 dims would leave the machine mostly idle
   A.par = (long long)L.n * ((A.nq + kDraftThreads - 1) / kDraftThreads) < 2ll * c->num_sms;
   const int per_block = A.par ? kDraftQ : kDraftThreads;
-  dim3 grid((A.nq + per_block - 1) / per_block, L.n);
+  dim3 grid(L.n, (A.nq + per_block - 1) / per_block);  // chains along x (no 65535 limit there)
   draft_kernel<<<grid, kDraftThreads, 0, c->stream>>>(A);
   c->launches++;
 }

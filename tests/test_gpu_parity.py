@@ -408,6 +408,33 @@ def test_degenerate_constant_drift_accepts_everything():
     assert res.rounds == 7 and rel_l2(y[0].cpu().numpy().astype(np.float64), res.y) < 1e-5
 
 
+def test_mixture_law_many_chains():
+    """cfg-1 statistical check on the GPU: 65536 ASD chains against 65536 sequential chains (other chain
+    ids) on the 8-component mixture - the two samplers have the same law (Theorem 3), compared per
+    coordinate (two-sample KS) and by nearest-component occupancy (chi-square)."""
+    from scipy import stats
+    n = 65536
+    wl = workloads.make("cfg1_gmm2d", chains=n)
+    with _sampler(wl) as s:
+        s.reset(n, 0)
+        ya, rounds, st = s.sample()
+        s.reset(n, n)
+        ys, _ = s.sequential_ddpm()
+    ya, ys = ya.cpu().numpy().astype(np.float64), ys.cpu().numpy().astype(np.float64)
+    _log(f"cfg1 n={n}: rounds mean {st.rounds_mean:.2f} max {st.rounds_max} of K={wl.K}")
+    T = wl.t[-1]
+    for j in range(2):
+        assert stats.ks_2samp(ya[:, j], ys[:, j]).pvalue > 1e-3
+    c = wl.means.astype(np.float64)
+    lab = lambda y: np.bincount(np.argmin(((y[:, None, :] / T - c[None]) ** 2).sum(-1), axis=1), minlength=len(c))
+    table = np.stack([lab(ya), lab(ys)])
+    table = table[:, table.sum(0) >= 20]
+    assert table.shape[1] >= 4 and stats.chi2_contingency(table)[1] > 1e-3
+    # every mode keeps mass: y_K / T lands within 4 component std + the 1/sqrt(T) blur of some mean
+    dist = np.sqrt(((ya[:, None, :] / T - c[None]) ** 2).sum(-1)).min(1)
+    assert np.mean(dist < 4 * (wl.sigma + 1 / math.sqrt(T))) > 0.99
+
+
 def test_gaussian_target_moments_many_chains():
     """cfg-2 statistical check on the GPU: 16384 ASD chains and 16384 sequential chains against the
     closed-form law of the Euler chain (mean T mu0, eigen-variances (1+T lam)^2 sum eta/(1+t lam)^2)."""
