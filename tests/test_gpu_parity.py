@@ -27,7 +27,7 @@ def _log(msg):
 
 # ------------------------------------------------------------------ drift alone
 @pytest.mark.parametrize("name,n_rows", [("cfg1_gmm2d", 100), ("gmm_odd", 57), ("gauss_small", 50),
-                                         ("cfg2_gauss64", 300), ("mlp_tiny", 23), ("mlp_ragged", 300),
+                                         ("cfg2_gauss64", 300), ("mlp_tiny", 23), ("mlp_odd", 19), ("mlp_odd", 300), ("mlp_ragged", 300),
                                          ("mlp_ragged", 1), ("mlp_ragged", 200), ("cfg3_policy", 17),
                                          ("cfg3_policy", 256), ("cfg3_policy", 400), ("cfg3_policy", 512), ("cfg3_policy", 700)])
 def test_drift_matches_oracle(name, n_rows):
@@ -131,7 +131,7 @@ def test_lockstep_bench_workload_sampled_chains():
 @pytest.mark.parametrize("all_slots", [False, True])
 @pytest.mark.parametrize("name,chains,rounds", [
     ("cfg1_gmm2d", 16, 60), ("gmm_odd", 9, 30), ("gauss_small", 11, 40), ("cfg2_gauss64", 24, 12),
-    ("mlp_tiny", 5, 25), ("mlp_ragged", 37, 8), ("cfg3_policy", 64, 3)])
+    ("mlp_tiny", 5, 25), ("mlp_odd", 7, 12), ("mlp_ragged", 37, 8), ("cfg3_policy", 64, 3)])
 def test_lockstep_rounds(name, chains, rounds, all_slots):
     """all_slots=False is the production path (the verify kernel stops at the first rejected slot);
     all_slots=True makes it evaluate the whole window so every ln ratio is compared."""

@@ -166,6 +166,9 @@ def make(name: str, *, chains: Optional[int] = None, K: Optional[int] = None,
     if name == "mlp_ragged":
         # odd sizes: d not a multiple of 8/16, in_dim padded, width spanning several N tiles
         return _mlp(name, 52, 12, 64, 320, 3, ov(K, 60), ov(window, 12), ov(chains, 37), s, bias_std=0.05)
+    if name == "mlp_odd":
+        # nothing a multiple of 4: scalar tails in draft / verify / epilogues, width of 72 = 9 x 8
+        return _mlp(name, 45, 3, 10, 72, 1, ov(K, 30), ov(window, 9), ov(chains, 7), s, bias_std=0.05)
     if name == "gmm_odd":
         return _gmm(name, 5, 3, 0.5, ov(K, 50), ov(window, 7), ov(chains, 9), s)
     if name == "gauss_small":
