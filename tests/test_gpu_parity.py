@@ -130,7 +130,7 @@ def test_lockstep_bench_workload_sampled_chains():
 # ------------------------------------------------------------------ lock-step rounds
 @pytest.mark.parametrize("all_slots", [False, True])
 @pytest.mark.parametrize("name,chains,rounds", [
-    ("cfg1_gmm2d", 16, 60), ("gmm_odd", 9, 30), ("gauss_small", 11, 40), ("cfg2_gauss64", 24, 12),
+    ("cfg1_gmm2d", 16, 60), ("gmm_odd", 9, 30), ("gmm_wide", 3, 6), ("gauss_small", 11, 40), ("cfg2_gauss64", 24, 12),
     ("mlp_tiny", 5, 25), ("mlp_odd", 7, 12), ("mlp_ragged", 37, 8), ("cfg3_policy", 64, 3)])
 def test_lockstep_rounds(name, chains, rounds, all_slots):
     """all_slots=False is the production path (the verify kernel stops at the first rejected slot);

@@ -169,6 +169,9 @@ def make(name: str, *, chains: Optional[int] = None, K: Optional[int] = None,
     if name == "mlp_odd":
         # nothing a multiple of 4: scalar tails in draft / verify / epilogues, width of 72 = 9 x 8
         return _mlp(name, 45, 3, 10, 72, 1, ov(K, 30), ov(window, 9), ov(chains, 7), s, bias_std=0.05)
+    if name == "gmm_wide":
+        # a wide, odd dimension: many float4 groups per row and a ragged tail in every kernel
+        return _gmm(name, 4099, 3, 0.5, ov(K, 12), ov(window, 6), ov(chains, 3), s, box=0.05)
     if name == "gmm_odd":
         return _gmm(name, 5, 3, 0.5, ov(K, 50), ov(window, 7), ov(chains, 9), s)
     if name == "gauss_small":
