@@ -308,6 +308,14 @@ asd_status asd_denoise_static(asd_ctx* ctx, int32_t n_rows, const int32_t* step_
                               const int32_t* slot_dev, float* out_dev);
 asd_status asd_denoise_static_max_rows(const asd_ctx* ctx, int32_t* max_rows_out);
 
+/*
+ * Failure-path self-test (the paper has no counterpart).  Every wait inside the kernels is bounded:
+ * when its limit (about 0.2 s) runs out the kernel records ASD_ERR_TIMEOUT, finishes, and the next
+ * synchronising call returns that status with the context still usable.  This call launches one thread
+ * that waits on a barrier nothing completes and returns what the library reports: ASD_ERR_TIMEOUT.
+ */
+asd_status asd_debug_wait_selftest(asd_ctx* ctx);
+
 /* Message for the last error on this context (static or context storage; never NULL). */
 const char* asd_last_error(const asd_ctx* ctx);
 

@@ -16,7 +16,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 EXPORTED_SYMBOLS = [
     "asd_version", "asd_create", "asd_reset", "asd_round", "asd_sample", "asd_sequential_ddpm",
     "asd_sample_host", "asd_get_state", "asd_set_state", "asd_get_window_state", "asd_set_window_state", "asd_debug_last_round", "asd_denoise",
-    "asd_set_profiling", "asd_get_profile", "asd_ddpm_schedule", "asd_denoise_static", "asd_denoise_static_max_rows",
+    "asd_set_profiling", "asd_get_profile", "asd_ddpm_schedule", "asd_debug_wait_selftest", "asd_denoise_static", "asd_denoise_static_max_rows",
     "asd_last_error", "asd_destroy",
 ]
 
@@ -136,6 +136,7 @@ def load_library():
         "asd_sample_host": [vp, i32, u64, vp, vp, i32, vp, vp, C.POINTER(_RunStats)],
         "asd_get_state": [vp, vp, vp, vp],
         "asd_set_state": [vp, vp, vp, vp],
+        "asd_debug_wait_selftest": [vp],
         "asd_ddpm_schedule": [i32, vp, i32, i32, i32, vp, vp, vp, vp, vp, vp],
         "asd_get_window_state": [vp, vp, vp],
         "asd_set_window_state": [vp, vp, vp],

@@ -981,6 +981,14 @@ asd_status asd_debug_last_round(asd_ctx* ctx, float* ln_ratio_dev, float* ln_u_d
   return ASD_OK;
 }
 
+asd_status asd_debug_wait_selftest(asd_ctx* ctx) {
+  if (!ctx) return ASD_ERR_INVALID_ARG;
+  Ctx* c = &ctx->c;
+  launch_wait_selftest(c);
+  ASD_CUDA(c, cudaGetLastError());
+  return sync_counters(c);  // reports and clears the device error word
+}
+
 asd_status asd_denoise(asd_ctx* ctx, int32_t n_rows, const int32_t* step_dev, const float* y_dev,
                        const int32_t* slot_dev, float* out_dev) {
   if (!ctx) return ASD_ERR_INVALID_ARG;

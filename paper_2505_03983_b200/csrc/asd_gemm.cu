@@ -926,6 +926,19 @@ gemm_skinny_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
   }
 }
 
+// Self-test of the bounded wait: one thread waits on a barrier that nothing will ever complete.  The
+// wait gives up after its limit, records ASD_ERR_TIMEOUT in the error word and the kernel returns.
+__global__ void wait_selftest_kernel(int* err) {
+  __shared__ uint64_t bar;
+  __shared__ int dead;
+  if (threadIdx.x == 0) {
+    mbar_init(smem_u32(&bar), 1);
+    dead = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    mbar_wait(smem_u32(&bar), 0u, &dead, err);
+  }
+}
+
 // ---- host side --------------------------------------------------------------------------------
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -1109,6 +1122,11 @@ asd_status launch_gemm(Ctx* c, const void* a_ptr, int a_cols, const void* w_ptr,
 }
 
 }  // namespace
+
+void launch_wait_selftest(Ctx* c) {
+  wait_selftest_kernel<<<1, 32, 0, c->stream>>>(&c->counters->err);
+  c->launches++;
+}
 
 asd_status mlp_forward(Ctx* c, const RowSet& rs, float* out, int pass) {
   const MlpParams& M = c->mlp;

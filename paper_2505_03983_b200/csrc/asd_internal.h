@@ -209,5 +209,6 @@ void launch_fill_int(Ctx* c, int* p, int n, int val);
 // Runs the GEMM chain on the rows already packed into mlp.X; writes out[r] for r < *n_rows_dev.
 // pass: 0 = drift at the current points, 1 = drift at the drafted points, 2 = stand-alone call.
 asd_status mlp_forward(Ctx* c, const RowSet& rs, float* out, int pass);
+void launch_wait_selftest(Ctx* c);  // one bounded wait that must run out (failure-path self-test)
 
 }  // namespace asd

@@ -435,6 +435,20 @@ def test_mixture_law_many_chains():
     assert np.mean(dist < 4 * (wl.sigma + 1 / math.sqrt(T))) > 0.99
 
 
+def test_bounded_wait_runs_out_and_context_survives():
+    """Failure path: a wait that nothing completes gives up after its limit, the call reports
+    ASD_ERR_TIMEOUT, and the same context then samples as before."""
+    wl = workloads.make("mlp_tiny")
+    with _sampler(wl) as s:
+        s.reset(wl.chains, 0, cond=wl.cond)
+        y0, r0, _ = s.sample()
+        st = s.lib.asd_debug_wait_selftest(s._ctx)
+        assert st == 6 and b"bounded" in s.lib.asd_last_error(s._ctx)        # ASD_ERR_TIMEOUT
+        s.reset(wl.chains, 0, cond=wl.cond)
+        y1, r1, _ = s.sample()
+    assert torch.equal(y0, y1) and torch.equal(r0, r1)
+
+
 def test_gaussian_target_moments_many_chains():
     """cfg-2 statistical check on the GPU: 16384 ASD chains and 16384 sequential chains against the
     closed-form law of the Euler chain (mean T mu0, eigen-variances (1+T lam)^2 sum eta/(1+t lam)^2)."""
