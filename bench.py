@@ -94,19 +94,26 @@ class ClockSampler:
 
 
 def oracle_sample_rate(wl, budget_s: float, max_rounds: int):
-    """Runs the oracle's ASD on chain 0 for at most `max_rounds` rounds / `budget_s` seconds and
-    returns (samples per second extrapolated by the fraction of the K steps covered, description)."""
+    """Runs the oracle's ASD chain after chain (at most `max_rounds` rounds each) until about
+    `budget_s` seconds have passed, and returns (samples per second, with an unfinished chain counted
+    by the fraction of its K steps, description)."""
     from oracle import asd as oasd, denoisers as oden
     g = oden.from_workload(wl)
     sch = oasd.make_schedule(wl.t)
-    y, a, rounds = np.zeros(wl.d), 0, 0
     t0 = time.perf_counter()
-    while a < wl.K and rounds < max_rounds and time.perf_counter() - t0 < budget_s:
-        rec = oasd.asd_round(g, sch, wl.seed, 0, 0, a, y, wl.window)
-        a, y, rounds = rec.a_after, rec.y_after, rounds + 1
+    done, chains, rounds_total = 0.0, 0, 0
+    while chains < wl.chains and (chains == 0 or time.perf_counter() - t0 < 0.5 * budget_s):
+        y, a, rounds = np.zeros(wl.d), 0, 0
+        slot = chains
+        while a < wl.K and rounds < max_rounds and time.perf_counter() - t0 < budget_s:
+            rec = oasd.asd_round(g, sch, wl.seed, slot, slot, a, y, wl.window)
+            a, y, rounds = rec.a_after, rec.y_after, rounds + 1
+        done += a / wl.K
+        chains += 1
+        rounds_total += rounds
     el = time.perf_counter() - t0
-    frac = a / wl.K
-    return frac / el, f"chain 0, first {rounds} rounds ({a} of {wl.K} steps) in {el:.1f} s, extrapolated by steps"
+    return done / el, (f"chains 0..{chains - 1}, {rounds_total} rounds = {done:.2f} samples' worth of steps in {el:.1f} s "
+                       f"(an unfinished chain counts by its fraction of the K steps)")
 
 
 def config_of(wl):
