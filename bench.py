@@ -306,8 +306,8 @@ def run_ours(args):
         "kernel": "verify_kernel (ASD_FLAG_DEBUG_ALL_SLOTS)", "bound": "hbm", "achieved": va, "peak": peaks["hbm_gbs"],
         "unit": "GB/s", "frac": va / peaks["hbm_gbs"], "launches": ver_all["launches"],
         "avg_launch_ms": ver_all["ms"] / max(ver_all["launches"], 1), "traffic": None,
-        "note": "6 rounds with every window slot verified: bytes = 4 d (w + 2) per chain-round, the figure BASELINE.json's "
-                "HBM target refers to; instruction issue (Philox + Box-Muller per element) bounds it, not HBM"}
+        "note": "6 rounds with every window slot verified: bytes = 4 d (w + 2) per chain-round (the whole-window "
+                "reading of the verify step); instruction issue (Philox + Box-Muller per element) bounds it, not HBM"}
     if wl.kind == "mlp":
         hid = prof["pass2_gemm_hidden"]
         flops = 2.0 * wl.width * wl.width * hid["rows"] * wl.n_layers       # all hidden-layer launches of pass 2
