@@ -189,6 +189,11 @@ asd_status asd_round(asd_ctx* ctx, asd_round_stats* stats_host);
  * the target is y_K / t_K); rounds_out_dev: [n] int32 or NULL; stats_host or NULL.
  * Synchronises the stream before returning.  Continues from the current state, so it may
  * follow asd_round / asd_set_state.
+ * The rounds are enqueued without waiting for one another (their counters come back through a pinned
+ * ring a few rounds late; rounds enqueued after the last chain finished do nothing) and, unless
+ * per-phase timing is on, each round is replayed as a CUDA graph on a stream of the library's own that
+ * is ordered after the work already in the context's stream and before what the caller enqueues after
+ * the call.  Do not call it (or asd_sequential_ddpm) while the context's stream is being captured.
  */
 asd_status asd_sample(asd_ctx* ctx, float* y_out_dev, int32_t* rounds_out_dev, asd_run_stats* stats_host);
 
