@@ -165,11 +165,18 @@ asd_status launch_captured(Ctx* c, const std::tuple<int, int, long long>& key, B
   return ASD_OK;
 }
 
-asd_status launch_round_graph(Ctx* c, int window, bool use_u, int active) {
+// `group` consecutive rounds in one graph: for the launch-bound workloads the graph launch itself is a
+// visible part of a round.
+asd_status launch_round_graph(Ctx* c, int window, bool use_u, int active, int group) {
   if (active <= 0) return ASD_OK;
   const int bucket = bound_bucket(c, active);
-  return launch_captured(c, std::make_tuple(window, use_u ? 1 : 0, (long long)bucket),
-                         [&] { return enqueue_round(c, window, use_u, bucket); });
+  return launch_captured(c, std::make_tuple(window, (use_u ? 1 : 0) + 16 * group, (long long)bucket), [&] {
+    for (int r = 0; r < group; ++r) {
+      const asd_status st = enqueue_round(c, window, use_u, bucket);
+      if (st != ASD_OK) return st;
+    }
+    return ASD_OK;
+  });
 }
 
 // One tick of the staggered schedule (network denoiser).  The batch is split into two lanes that run
@@ -245,8 +252,16 @@ struct PrivateStreamScope {
   }
 };
 
-asd_status enqueue_round_any(Ctx* c, bool graphs, int window, bool use_u, int active) {
-  return graphs ? launch_round_graph(c, window, use_u, active) : enqueue_round(c, window, use_u, active);
+constexpr int kRoundsPerGraph = 4;
+
+// `group` rounds: one graph replay, or the kernels themselves
+asd_status enqueue_rounds(Ctx* c, bool graphs, int window, bool use_u, int active, int group) {
+  if (graphs) return launch_round_graph(c, window, use_u, active, group);
+  for (int r = 0; r < group; ++r) {
+    const asd_status st = enqueue_round(c, window, use_u, active);
+    if (st != ASD_OK) return st;
+  }
+  return ASD_OK;
 }
 
 // Whether asd_sample runs the batch as two staggered lanes (network denoiser only).  Off unless
@@ -818,11 +833,15 @@ asd_status asd_sample(asd_ctx* ctx, float* y_out_dev, int32_t* rounds_out_dev, a
     ++consumed;
     return true;
   };
-  while (active > 0 && issued < max_rounds && deferred == ASD_OK) {
+  // with graph replay a ring slot stands for kRoundsPerGraph rounds (the counters of the last one)
+  // (fewer when the run is short: rounds enqueued after the last chain finished are wasted launches)
+  const int min_rounds = (c->K + c->window - 1) / c->window;
+  const int group = pss.on ? std::max(1, std::min(kRoundsPerGraph, min_rounds / 16)) : 1;
+  while (active > 0 && issued * group < max_rounds + group && deferred == ASD_OK) {
     const int slot = (int)(issued % Ctx::kRing);
     c->ev_used = (size_t)slot * kEventsPerRound;
     const size_t pending0 = c->pending.size();
-    asd_status st = enqueue_round_any(c, pss.on, c->window, true, active);
+    asd_status st = enqueue_rounds(c, pss.on, c->window, true, active, group);
     if (st != ASD_OK) return st;
     prof_pairs[slot] = c->pending.size() - pending0;
     ASD_CUDA(c, cudaMemcpyAsync(&c->ring_host[slot], c->counters, sizeof(RoundCounters), cudaMemcpyDeviceToHost, c->stream));
@@ -859,9 +878,11 @@ asd_status asd_sequential_ddpm(asd_ctx* ctx, float* y_out_dev, asd_run_stats* st
   ASD_CUDA(c, cudaEventRecord(c->ev0, c->stream));
   {
     PrivateStreamScope pss(c);
-    for (int i = min_a; i < c->K; ++i) {
-      asd_status st = enqueue_round_any(c, pss.on, 1, false, c->n);
+    for (int i = min_a; i < c->K;) {
+      const int group = (pss.on && c->K - i >= kRoundsPerGraph) ? kRoundsPerGraph : 1;
+      asd_status st = enqueue_rounds(c, pss.on, 1, false, c->n, group);
       if (st != ASD_OK) return st;
+      i += group;
     }
   }
   return finish_run(c, y_out_dev, nullptr, stats_host, launches0, true);
