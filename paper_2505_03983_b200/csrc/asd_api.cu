@@ -725,6 +725,7 @@ asd_status asd_reset(asd_ctx* ctx, int32_t n_chains, uint64_t chain_id_base, con
   }
   ASD_CUDA(c, cudaGetLastError());
   c->have_reset = true;
+  c->round_bound = n_chains;
   c->launches = 0;
   return ASD_OK;
 }
@@ -733,12 +734,14 @@ asd_status asd_round(asd_ctx* ctx, asd_round_stats* stats_host) {
   if (!ctx) return ASD_ERR_INVALID_ARG;
   Ctx* c = &ctx->c;
   if (!c->have_reset) return fail(c, ASD_ERR_STATE, "asd_round before asd_reset");
-  asd_status st = enqueue_round(c, c->window, true, c->n);
+  // the bound on the active chains that sizes the grids: what the previous round reported, if it was read
+  asd_status st = enqueue_round(c, c->window, true, std::min(c->n, c->round_bound));
   if (st != ASD_OK) return st;
   if (stats_host) {
     st = sync_counters(c);
     if (st != ASD_OK) return st;
     const RoundCounters& h = *c->counters_host;
+    c->round_bound = std::max(h.n_active_after, 1);
     stats_host->n_active_before = h.n_active;
     stats_host->n_active_after = h.n_active_after;
     stats_host->rows_pass1 = h.n_active;
@@ -965,7 +968,10 @@ asd_status asd_set_state(asd_ctx* ctx, const int32_t* a_dev, const float* y_dev,
   if (!ctx) return ASD_ERR_INVALID_ARG;
   Ctx* c = &ctx->c;
   if (!c->have_reset) return fail(c, ASD_ERR_STATE, "asd_set_state before asd_reset");
-  if (a_dev) ASD_CUDA(c, cudaMemcpyAsync(c->a, a_dev, (size_t)c->n * sizeof(int), cudaMemcpyDeviceToDevice, c->stream));
+  if (a_dev) {
+    ASD_CUDA(c, cudaMemcpyAsync(c->a, a_dev, (size_t)c->n * sizeof(int), cudaMemcpyDeviceToDevice, c->stream));
+    c->round_bound = c->n;  // cursors may have moved back: every chain may be active again
+  }
   if (y_dev) ASD_CUDA(c, cudaMemcpyAsync(c->y, y_dev, (size_t)c->n * c->d * sizeof(float), cudaMemcpyDeviceToDevice, c->stream));
   if (rounds_dev)
     ASD_CUDA(c, cudaMemcpyAsync(c->rounds, rounds_dev, (size_t)c->n * sizeof(int), cudaMemcpyDeviceToDevice, c->stream));

@@ -118,6 +118,7 @@ struct Ctx {
   int n = 0;  // chains of the current reset
   uint64_t chain_base = 0;
   bool have_reset = false;
+  int round_bound = 0;  // asd_round: upper bound on the active chains (chains only finish, so a stale value is valid)
   bool adaptive = false;         // ASD_FLAG_ADAPTIVE_WINDOW
   bool debug_all_slots = false;  // ASD_FLAG_DEBUG_ALL_SLOTS: the verify kernel evaluates every window slot
   // device arrays
