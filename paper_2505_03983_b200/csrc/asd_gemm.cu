@@ -179,7 +179,7 @@ __device__ __forceinline__ void mbar_arrive_cluster(uint32_t bar_cluster_addr) {
   asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(bar_cluster_addr) : "memory");
 }
 // TMA load into this CTA's shared memory whose completion bytes are counted on a barrier of either
-// CTA of the pair (no multicast: every CTA fetches its own box).
+// CTA of the pair (every CTA fetches its own box).
 __device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, uint32_t bar_cluster_addr, int x,
                                                  int y) {
   asm volatile(
