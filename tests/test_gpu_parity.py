@@ -252,6 +252,33 @@ def test_staggered_lanes_equal_plain_rounds(name, chains, window, graphs, monkey
     assert st0.rounds_mean == st1.rounds_mean and torch.isfinite(y1).all()
 
 
+@pytest.mark.parametrize("case", range(12))
+def test_lockstep_random_small_shapes(case):
+    """Seeded random shapes (dimension, grid length, window, batch, network sizes) of all three drift kinds,
+    a few lock-step rounds each, with and without per-chain adaptive windows."""
+    from paper_2505_03983_b200.binding import FLAG_ADAPTIVE_WINDOW
+    rng = np.random.default_rng(1000 + case)
+    kind = ("gmm", "gauss", "mlp")[case % 3]
+    K, window, chains = int(rng.integers(3, 70)), int(rng.integers(2, 65)), int(rng.integers(1, 40))
+    if kind == "gmm":
+        wl = workloads._gmm(f"rand{case}", int(rng.integers(1, 300)), int(rng.integers(1, 6)), 0.4, K, window, chains,
+                            case, box=1.0)
+    elif kind == "gauss":
+        wl = workloads._gauss(f"rand{case}", int(rng.integers(1, 90)), K, window, chains, case)
+    else:
+        wl = workloads._mlp(f"rand{case}", int(rng.integers(1, 200)), int(rng.integers(0, 20)), 2 * int(rng.integers(0, 20)),
+                            8 * int(rng.integers(1, 40)), int(rng.integers(0, 4)), K, window, chains, case, bias_std=0.05)
+    cond = wl.cond if wl.kind == "mlp" and wl.d_cond else None
+    adaptive = bool(case & 1)
+    with _sampler(wl, flags=FLAG_ADAPTIVE_WINDOW if adaptive else 0) as s:
+        worst = lockstep(s, wl, chains, 6, chain_base=case * 100, cond=cond, log=_log, adaptive=adaptive)
+        s.reset(chains, case * 100, cond=cond)
+        y, r, st = s.sample()
+    assert torch.isfinite(y).all() and int(r.min()) >= 1 and worst["rounds"] >= 1
+    _log(f"random case {case}: {kind} d={wl.d} K={K} window={window} chains={chains} adaptive={adaptive} "
+         f"rounds mean {st.rounds_mean:.1f}")
+
+
 def test_lockstep_window_64_and_window_beyond_K():
     from paper_2505_03983_b200.binding import FLAG_DEBUG_ALL_SLOTS
     wl = workloads.make("gauss_small", K=70, window=64, chains=6)
