@@ -235,7 +235,7 @@ def run_ours(args):
     _, st_seq = s.sequential_ddpm()
     s.close()
     # ---- the verify kernel when it evaluates the whole window (Algorithm 2 as written) ---------------
-    from paper_2505_03983_b200.binding import FLAG_ADAPTIVE_WINDOW, FLAG_DEBUG_ALL_SLOTS
+    from paper_2505_03983_b200.binding import FLAG_ADAPTIVE_WINDOW, FLAG_DEBUG_ALL_SLOTS, FLAG_LOOKAHEAD
     sv = AsdSampler(wl, flags=FLAG_DEBUG_ALL_SLOTS)
     sv.reset(n, base, cond=cond_dev)
     for _ in range(2):
@@ -247,27 +247,33 @@ def run_ours(args):
         all_rows += st_r.rows_pass2; all_chains += st_r.n_active_before
     ver_all = sv.get_profile()["verify"]
     sv.close()
-    sa = AsdSampler(wl, flags=FLAG_ADAPTIVE_WINDOW)
-    for _ in range(2):
-        sa.reset(n, base, cond=cond_dev)
-        sa.sample()
-    barrier()
-    a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    a0.record()
-    ad_rounds, ad_rows = [], 0
-    for _ in range(args.steps):
-        sa.reset(n, base, cond=cond_dev)
-        _, _, st_a = sa.sample()
-        ad_rounds.append(st_a.rounds_mean); ad_rows += st_a.rows_total
-    a1.record()
-    barrier()
-    ms_adapt = a0.elapsed_time(a1)
-    sa.close()
+    def timed_variant(flags):
+        """The same steps on a sampler created with `flags`: (ms, mean rounds per sample, drift rows)."""
+        sx = AsdSampler(wl, flags=flags)
+        for _ in range(2):
+            sx.reset(n, base, cond=cond_dev)
+            sx.sample()
+        barrier()
+        x0, x1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        x0.record()
+        rnds, nrows = [], 0
+        for _ in range(args.steps):
+            sx.reset(n, base, cond=cond_dev)
+            _, _, st_x = sx.sample()
+            rnds.append(st_x.rounds_mean); nrows += st_x.rows_total
+        x1.record()
+        barrier()
+        sx.close()
+        return x0.elapsed_time(x1), float(np.mean(rnds)), nrows
 
-    t = torch.tensor([ms, ms_e2e, st_seq.ms_total, ms_plain, ms_adapt], dtype=torch.float64, device="cuda")
+    ms_adapt, ad_rounds, ad_rows = timed_variant(FLAG_ADAPTIVE_WINDOW)
+    ms_la, la_rounds, la_rows = timed_variant(FLAG_LOOKAHEAD)
+    ms_ala, ala_rounds, ala_rows = timed_variant(FLAG_ADAPTIVE_WINDOW | FLAG_LOOKAHEAD)
+
+    t = torch.tensor([ms, ms_e2e, st_seq.ms_total, ms_plain, ms_adapt, ms_la, ms_ala], dtype=torch.float64, device="cuda")
     if dist is not None:
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms, ms_e2e, ms_seq, ms_plain, ms_adapt = [float(x) for x in t.cpu()]
+    ms, ms_e2e, ms_seq, ms_plain, ms_adapt, ms_la, ms_ala = [float(x) for x in t.cpu()]
     if rank != 0:
         if dist is not None:
             dist.destroy_process_group()
@@ -293,10 +299,17 @@ def run_ours(args):
                            "wallclock_speedup_asd": (ms_seq) / (ms / args.steps)},
         "without_phase_events": {"value": total / (ms_plain / 1e3), "unit": UNIT, "ms_per_step": ms_plain / args.steps},
         "adaptive_window": {"value": total / (ms_adapt / 1e3), "unit": UNIT, "ms_per_step": ms_adapt / args.steps,
-                            "rounds_per_sample": float(np.mean(ad_rounds)),
+                            "rounds_per_sample": ad_rounds,
                             "drift_rows_per_sample_over_K": ad_rows / (args.steps * n * wl.K),
                             "note": "same workload, every chain picks its speculation length in 2..window from its "
                                     "own acceptance history (ASD_FLAG_ADAPTIVE_WINDOW); CUDA-graph rounds"},
+        "lookahead": {"value": total / (ms_la / 1e3), "unit": UNIT, "ms_per_step": ms_la / args.steps,
+                      "rounds_per_sample": la_rounds, "drift_rows_per_sample_over_K": la_rows / (args.steps * n * wl.K),
+                      "note": "same workload with ASD_FLAG_LOOKAHEAD: the batched pass also evaluates the end of the "
+                              "window, and a chain that accepted its whole window skips its next first model call"},
+        "adaptive_window_lookahead": {"value": total / (ms_ala / 1e3), "unit": UNIT, "ms_per_step": ms_ala / args.steps,
+                                      "rounds_per_sample": ala_rounds,
+                                      "drift_rows_per_sample_over_K": ala_rows / (args.steps * n * wl.K)},
         "phases_ms": {k: round(v["ms"], 3) for k, v in prof.items() if v["launches"]},
     }
     # ---- roofline of the dominant kernel ----------------------------------------------------

@@ -137,6 +137,19 @@ typedef struct {
  */
 #define ASD_FLAG_ADAPTIVE_WINDOW 2u
 
+/*
+ * ASD_FLAG_LOOKAHEAD: the batched pass also evaluates the drift at the LAST drafted point of each
+ * window, y^_{a+w} (when a + w < K).  If the whole window is accepted that point is the chain's next
+ * state and the drift there is exactly the v_a that the next iteration of Algorithm 1 would compute in
+ * its first model call, so the call is skipped: a round then costs one sequential model pass instead of
+ * two for every chain that accepted its window.  The law of the output is untouched (the same function
+ * is evaluated at the same point, one round earlier); per-chain results agree with the default mode
+ * up to the rounding differences of evaluating that row inside a different batch.  Costs one more row
+ * per chain and round in the batched pass and a [max_chains, d] float buffer.  rows_pass1 then counts
+ * only the chains whose first call was really made.
+ */
+#define ASD_FLAG_LOOKAHEAD 4u
+
 typedef struct {
   int32_t n_active_before; /* chains with a < K when the round started */
   int32_t n_active_after;

@@ -25,6 +25,7 @@ STATUS = {0: "ASD_OK", 1: "ASD_ERR_INVALID_ARG", 2: "ASD_ERR_UNSUPPORTED", 3: "A
 KIND = {"gmm": 0, "gauss": 1, "mlp": 2}
 FLAG_DEBUG_ALL_SLOTS = 1   # ASD_FLAG_DEBUG_ALL_SLOTS
 FLAG_ADAPTIVE_WINDOW = 2   # ASD_FLAG_ADAPTIVE_WINDOW
+FLAG_LOOKAHEAD = 4         # ASD_FLAG_LOOKAHEAD
 
 
 PRED = {"x0": 0, "eps": 1, "v": 2}

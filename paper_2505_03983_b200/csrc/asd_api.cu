@@ -82,8 +82,13 @@ asd_status enqueue_round(Ctx* c, int window, bool use_u, int active_bound) {
     ProfScope ps(c, PH_PREP);
     launch_prep(c, whole_batch(c), window);
   }
-  RowSet rs1{&c->counters->n_active, active_bound, c->y, c->act, c->step1, c->act};
-  RowSet rs2{&c->counters->rows2, active_bound * (window - 1), c->Yhat, nullptr, c->row_step, c->row_slot};
+  // look-ahead: the first model call covers only the chains without a saved drift, and every chain may
+  // draft one more row (the point the next round would start from)
+  const bool la = c->lookahead;
+  RowSet rs1{la ? &c->counters->n_eval : &c->counters->n_active, active_bound, c->y, la ? c->act1 : c->act,
+             la ? c->step1e : c->step1, la ? c->act1 : c->act, true};
+  RowSet rs2{&c->counters->rows2, active_bound * (la ? window : window - 1), c->Yhat, nullptr, c->row_step, c->row_slot,
+             true};  // both counts come from the prep kernel; a pack or draft kernel runs in between
   asd_status st = ASD_OK;
   switch (c->kind) {
     case ASD_DEN_GMM_ISO:
@@ -270,7 +275,7 @@ asd_status enqueue_rounds(Ctx* c, bool graphs, int window, bool use_u, int activ
 // and the doubled draft / verify launches (936 against 920 ms and 3583 against 3545 ms per step); the
 // run is bound by the power cap, so what counts is energy per FLOP, not idle gaps.
 bool use_stagger(const Ctx* c) {
-  if (c->kind != ASD_DEN_RESMLP_BF16 || !c->G2 || c->window < 4 || c->n < 2) return false;
+  if (c->kind != ASD_DEN_RESMLP_BF16 || !c->G2 || c->window < 4 || c->n < 2 || c->lookahead) return false;
   const char* e = getenv("ASD_STAGGER");
   return e && e[0] == '1';
 }
@@ -454,7 +459,7 @@ asd_status asd_create(const asd_config* cfg, void* cuda_stream, asd_ctx** out) {
   if (cfg->K < 1) return bad(ASD_ERR_INVALID_ARG, "K must be >= 1");
   if (cfg->window < 1 || cfg->window > kMaxWindow) return bad(ASD_ERR_INVALID_ARG, "window must be in 1..64");
   if (cfg->max_chains < 1) return bad(ASD_ERR_INVALID_ARG, "max_chains must be >= 1");
-  if (cfg->flags & ~(ASD_FLAG_DEBUG_ALL_SLOTS | ASD_FLAG_ADAPTIVE_WINDOW)) return bad(ASD_ERR_INVALID_ARG, "unknown flag");
+  if (cfg->flags & ~(ASD_FLAG_DEBUG_ALL_SLOTS | ASD_FLAG_ADAPTIVE_WINDOW | ASD_FLAG_LOOKAHEAD)) return bad(ASD_ERR_INVALID_ARG, "unknown flag");
   if (!cfg->t) return bad(ASD_ERR_INVALID_ARG, "t must not be NULL");
   if (!(cfg->t[0] >= 0.0)) return bad(ASD_ERR_INVALID_ARG, "t[0] must be >= 0");
   for (int i = 0; i < cfg->K; ++i) {
@@ -463,7 +468,8 @@ asd_status asd_create(const asd_config* cfg, void* cuda_stream, asd_ctx** out) {
     if (cfg->sigma2 && !(cfg->sigma2[i] > 0.0 && isfinite(cfg->sigma2[i])))
       return bad(ASD_ERR_INVALID_ARG, "sigma2 must be finite and positive");
   }
-  const long long max_rows_ll = (long long)cfg->max_chains * std::max(cfg->window - 1, 1);
+  const bool lookahead = (cfg->flags & ASD_FLAG_LOOKAHEAD) != 0;
+  const long long max_rows_ll = (long long)cfg->max_chains * (lookahead ? cfg->window : std::max(cfg->window - 1, 1));
   if (max_rows_ll > (1ll << 30) || max_rows_ll * cfg->d > (1ll << 40))
     return bad(ASD_ERR_INVALID_ARG, "max_chains * window * d too large");
   const asd_denoiser& D = cfg->den;
@@ -509,7 +515,8 @@ asd_status asd_create(const asd_config* cfg, void* cuda_stream, asd_ctx** out) {
   c->debug_all_slots = (cfg->flags & ASD_FLAG_DEBUG_ALL_SLOTS) != 0;
   c->adaptive = (cfg->flags & ASD_FLAG_ADAPTIVE_WINDOW) != 0;
   c->stream = static_cast<cudaStream_t>(cuda_stream);
-  c->max_rows = (int)((long long)cfg->max_chains * std::max(c->window - 1, 1));
+  c->lookahead = lookahead;
+  c->max_rows = (int)((long long)cfg->max_chains * (lookahead ? c->window : std::max(c->window - 1, 1)));
   cudaGetDevice(&c->device);
   cudaDeviceProp prop;
   if (cudaGetDeviceProperties(&prop, c->device) != cudaSuccess) return abandon(fail(c, ASD_ERR_CUDA, "device query failed"));
@@ -584,6 +591,13 @@ asd_status asd_create(const asd_config* cfg, void* cuda_stream, asd_ctx** out) {
   TRY(dev_alloc(c, &c->dbg_lr, n * c->window));
   TRY(dev_alloc(c, &c->dbg_lu, n * c->window));
   TRY(dev_alloc(c, &c->acc_len, n));
+  if (c->lookahead) {
+    TRY(dev_alloc(c, &c->has_v, n));
+    TRY(dev_alloc(c, &c->vsave, n * d));
+    TRY(dev_alloc(c, &c->act1, n));
+    TRY(dev_alloc(c, &c->step1e, n));
+    TRY(dev_alloc(c, &c->idx1, n));
+  }
   TRY(dev_alloc(c, &c->counters, 2));  // [0] round counters, [1].n_active doubles as a row-count scratch
 
   // ---- denoiser parameters ---------------------------------------------------------------------
@@ -703,6 +717,7 @@ asd_status asd_reset(asd_ctx* ctx, int32_t n_chains, uint64_t chain_id_base, con
   ASD_CUDA(c, cudaMemsetAsync(c->rounds, 0, (size_t)c->max_chains * sizeof(int), c->stream));
   ASD_CUDA(c, cudaMemsetAsync(c->counters, 0, 2 * sizeof(RoundCounters), c->stream));
   launch_fill_int(c, c->acc_len, c->max_chains, -1);
+  if (c->has_v) ASD_CUDA(c, cudaMemsetAsync(c->has_v, 0, (size_t)c->max_chains * sizeof(int), c->stream));
   if (c->G2) {
     const int h = (n_chains + 1) / 2;
     c->lanes[0].start = 0;
@@ -744,7 +759,7 @@ asd_status asd_round(asd_ctx* ctx, asd_round_stats* stats_host) {
     c->round_bound = std::max(h.n_active_after, 1);
     stats_host->n_active_before = h.n_active;
     stats_host->n_active_after = h.n_active_after;
-    stats_host->rows_pass1 = h.n_active;
+    stats_host->rows_pass1 = c->lookahead ? h.n_eval : h.n_active;
     stats_host->rows_pass2 = h.rows2;
     stats_host->accepted_total = (int64_t)h.accepted;
   }
@@ -828,9 +843,9 @@ asd_status asd_sample(asd_ctx* ctx, float* y_out_dev, int32_t* rounds_out_dev, a
     active = h.n_active_after;
     if (c->prof_on) {
       prof_collect_some(c, (long long)prof_pairs[slot]);
-      const long long n1 = h.n_active, n2 = h.rows2;
-      for (int ph : {PH_PREP, PH_PACK, PH_D1_IN, PH_D1_HID, PH_D1_OUT, PH_D1_ANALYTIC, PH_DRAFT, PH_VERIFY})
-        c->prof[ph].rows += n1;
+      const long long n1 = h.n_active, n1e = c->lookahead ? h.n_eval : h.n_active, n2 = h.rows2;
+      for (int ph : {PH_PREP, PH_DRAFT, PH_VERIFY}) c->prof[ph].rows += n1;
+      for (int ph : {PH_PACK, PH_D1_IN, PH_D1_HID, PH_D1_OUT, PH_D1_ANALYTIC}) c->prof[ph].rows += n1e;
       for (int ph : {PH_D2_IN, PH_D2_HID, PH_D2_OUT, PH_D2_ANALYTIC}) c->prof[ph].rows += n2;
     }
     ++consumed;
@@ -973,6 +988,8 @@ asd_status asd_set_state(asd_ctx* ctx, const int32_t* a_dev, const float* y_dev,
     c->round_bound = c->n;  // cursors may have moved back: every chain may be active again
   }
   if (y_dev) ASD_CUDA(c, cudaMemcpyAsync(c->y, y_dev, (size_t)c->n * c->d * sizeof(float), cudaMemcpyDeviceToDevice, c->stream));
+  // a saved drift belongs to the point and step it was evaluated at
+  if ((a_dev || y_dev) && c->has_v) ASD_CUDA(c, cudaMemsetAsync(c->has_v, 0, (size_t)c->max_chains * sizeof(int), c->stream));
   if (rounds_dev)
     ASD_CUDA(c, cudaMemcpyAsync(c->rounds, rounds_dev, (size_t)c->n * sizeof(int), cudaMemcpyDeviceToDevice, c->stream));
   return ASD_OK;

@@ -39,6 +39,7 @@ struct GemmArgs {
   int n_out;            // N
   int k_dim;            // K (any; the TMA zero-fills beyond the tensor)
   const int* m_dev;     // valid rows (device)
+  int m_settled;        // *m_dev was final before the kernel in front of this chain started (see RowSet)
   int m_cap;            // rows of the activation buffers
   const float* bias;    // [N]
   __nv_bfloat16* out_bf16;        // EPI_IN / EPI_HID: [m, ld_h]
@@ -768,6 +769,15 @@ gemm_skinny_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
   // grid_dependency_wait() below.  The weights do not, so their first tiles are fetched before it.
   grid_launch_dependents();
 
+  // A row block without a single valid row has nothing to compute or store: its cluster leaves before it
+  // streams any weights (a pass over zero rows, or a grid sized for a bound above the real count).  It still
+  // waits for the previous kernel, so that "this kernel has completed" keeps implying that every kernel
+  // before it has.
+  if (g.m_settled && min(__ldcg(g.m_dev), g.m_cap) <= row0) {
+    grid_dependency_wait();
+    return;
+  }
+
   if (threadIdx.x == 0) {
     prefetch_tmap(&map_x);
     prefetch_tmap(&map_w);
@@ -1144,6 +1154,7 @@ asd_status mlp_forward(Ctx* c, const RowSet& rs, float* out, int pass) {
   if (m_bound <= 0) return ASD_OK;
   GemmArgs g{};
   g.m_dev = rs.n_rows_dev;
+  g.m_settled = rs.settled ? 1 : 0;
   g.m_cap = M.row_cap;
   g.err = &c->counters->err;
   asd_status st;

@@ -28,7 +28,8 @@ struct RoundCounters {
   unsigned long long accepted;  // steps advanced this round
   unsigned long long rows_total;  // running total of drift evaluations since reset
   unsigned long long rows_verified;  // running total of drift rows the verify kernel read since reset
-  unsigned long long pad[1];
+  int n_eval;                   // chains whose v_a has to be evaluated this round (look-ahead: not all active ones)
+  int pad;
 };
 
 // Per-step fp32 tables, built on the host in fp64 (asd_create).
@@ -52,6 +53,10 @@ struct RowSet {
   const int* row_map;
   const int* row_step;
   const int* row_slot;
+  // true when *n_rows_dev was written by a kernel (or copy) that had completed before the kernel directly in
+  // front of the consumer started, so a kernel launched with programmatic stream serialization may read it
+  // before its dependency wait
+  bool settled = false;
 };
 
 struct GmmParams {
@@ -93,6 +98,11 @@ struct Lane {
   int* step1 = nullptr;      // [n]
   RoundCounters* counters = nullptr;
   int* v_off = nullptr;      // device int: row of the drift buffer where this lane's v_a rows start
+  // look-ahead (whole batch only): chains that need the first model call, their steps, and for every
+  // active position the row of that call's output (or -1: v_a was saved by the previous round)
+  int* act1 = nullptr;
+  int* step1e = nullptr;
+  int* idx1 = nullptr;
 };
 
 // Phases of a round, for the optional per-phase CUDA-event timing.
@@ -120,6 +130,12 @@ struct Ctx {
   bool have_reset = false;
   int round_bound = 0;  // asd_round: upper bound on the active chains (chains only finish, so a stale value is valid)
   bool adaptive = false;         // ASD_FLAG_ADAPTIVE_WINDOW
+  bool lookahead = false;        // ASD_FLAG_LOOKAHEAD
+  int* has_v = nullptr;          // [max_chains] 1: vsave holds v_a of the chain's next round
+  float* vsave = nullptr;        // [max_chains, d]
+  int* act1 = nullptr;           // [max_chains]
+  int* step1e = nullptr;         // [max_chains]
+  int* idx1 = nullptr;           // [max_chains]
   bool debug_all_slots = false;  // ASD_FLAG_DEBUG_ALL_SLOTS: the verify kernel evaluates every window slot
   // device arrays
   float* y = nullptr;        // [max_chains, d]

@@ -118,70 +118,90 @@ __device__ __forceinline__ float warp_sum(float x) {
 // Round driver bookkeeping: compact the chains with a < K into the active list and lay out the
 // pass-2 rows (exclusive scan of w - 1).  One block; n is at most a few tens of thousands.
 // ---------------------------------------------------------------------------------------------
+// Rows a chain drafts: its window minus the last slot (rebuilt by the verify kernel), plus - with
+// look-ahead - that last slot after all, when there is a step beyond it whose drift it can supply.
+__device__ __forceinline__ int drafted_rows(int w, int a, int K, int la) { return w - 1 + ((la && a + w < K) ? 1 : 0); }
+
 __global__ void __launch_bounds__(1024) prep_kernel(const int* __restrict__ a, const int* __restrict__ wnd, int n, int K,
-                                                    int window,
+                                                    int window, const int* __restrict__ has_v, int la,
                                                     int* __restrict__ act, int* __restrict__ row_off,
-                                                    int* __restrict__ step1, int* __restrict__ acc_len,
-                                                    RoundCounters* __restrict__ cnt) {
-  __shared__ int s_cnt[32], s_rows[32];
-  __shared__ int s_base_cnt, s_base_rows;
+                                                    int* __restrict__ step1, int* __restrict__ act1,
+                                                    int* __restrict__ step1e, int* __restrict__ idx1,
+                                                    int* __restrict__ acc_len, RoundCounters* __restrict__ cnt) {
+  __shared__ int s_cnt[32], s_rows[32], s_ev[32];
+  __shared__ int s_base_cnt, s_base_rows, s_base_ev;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   if (tid == 0) {
     s_base_cnt = 0;
     s_base_rows = 0;
+    s_base_ev = 0;
   }
   __syncthreads();
   for (int j0 = 0; j0 < n; j0 += blockDim.x) {
     const int j = j0 + tid;
-    int aj = K, flag = 0, rows = 0;
+    int aj = K, flag = 0, rows = 0, ev = 0;
     if (j < n) {
       aj = a[j];
       flag = aj < K;
-      rows = flag ? chain_window(wnd, j, window, K, aj) - 1 : 0;
+      rows = flag ? drafted_rows(chain_window(wnd, j, window, K, aj), aj, K, la) : 0;
+      ev = flag && !(la && has_v[j]);  // v_a still has to be evaluated
       acc_len[j] = -1;
     }
     // inclusive warp scans
-    int c = flag, r = rows;
+    int c = flag, r = rows, e = ev;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
       const int c2 = __shfl_up_sync(0xffffffffu, c, o);
       const int r2 = __shfl_up_sync(0xffffffffu, r, o);
+      const int e2 = __shfl_up_sync(0xffffffffu, e, o);
       if (lane >= o) {
         c += c2;
         r += r2;
+        e += e2;
       }
     }
     if (lane == 31) {
       s_cnt[warp] = c;
       s_rows[warp] = r;
+      s_ev[warp] = e;
     }
     __syncthreads();
     if (warp == 0) {
-      int wc = s_cnt[lane], wr = s_rows[lane];
+      int wc = s_cnt[lane], wr = s_rows[lane], we = s_ev[lane];
 #pragma unroll
       for (int o = 1; o < 32; o <<= 1) {
         const int c2 = __shfl_up_sync(0xffffffffu, wc, o);
         const int r2 = __shfl_up_sync(0xffffffffu, wr, o);
+        const int e2 = __shfl_up_sync(0xffffffffu, we, o);
         if (lane >= o) {
           wc += c2;
           wr += r2;
+          we += e2;
         }
       }
       s_cnt[lane] = wc;
       s_rows[lane] = wr;
+      s_ev[lane] = we;
     }
     __syncthreads();
     const int pos = s_base_cnt + (warp ? s_cnt[warp - 1] : 0) + c - flag;
     const int roff = s_base_rows + (warp ? s_rows[warp - 1] : 0) + r - rows;
+    const int epos = s_base_ev + (warp ? s_ev[warp - 1] : 0) + e - ev;
     if (flag) {
       act[pos] = j;
       row_off[pos] = roff;
       step1[pos] = aj;
+      if (idx1) idx1[pos] = ev ? epos : -1;
+      if (ev && act1) {
+        act1[epos] = j;
+        step1e[epos] = aj;
+      }
     }
     __syncthreads();
     if (tid == 0) {
       s_base_cnt += s_cnt[31];
       s_base_rows += s_rows[31];
+      s_base_ev += s_ev[31];
     }
     __syncthreads();
   }
@@ -189,9 +209,10 @@ __global__ void __launch_bounds__(1024) prep_kernel(const int* __restrict__ a, c
     row_off[s_base_cnt] = s_base_rows;
     cnt->n_active = s_base_cnt;
     cnt->rows2 = s_base_rows;
+    cnt->n_eval = s_base_ev;
     cnt->n_active_after = 0;
     cnt->accepted = 0ull;
-    cnt->rows_total += (unsigned long long)(s_base_cnt + s_base_rows);
+    cnt->rows_total += (unsigned long long)(s_base_ev + s_base_rows);
   }
 }
 
@@ -206,13 +227,18 @@ Lane whole_batch(const Ctx* c) {
   L.row_off = c->row_off;
   L.step1 = c->step1;
   L.counters = c->counters;
+  L.act1 = c->act1;
+  L.step1e = c->step1e;
+  L.idx1 = c->idx1;
   return L;
 }
 
 void launch_prep(Ctx* c, const Lane& L, int window) {
   const int* wnd = round_windows(c, window);
-  prep_kernel<<<1, 1024, 0, c->stream>>>(c->a + L.start, wnd ? wnd + L.start : nullptr, L.n, c->K, window, L.act, L.row_off,
-                                         L.step1, c->acc_len + L.start, L.counters);
+  const int la = (c->lookahead && L.act1) ? 1 : 0;
+  prep_kernel<<<1, 1024, 0, c->stream>>>(c->a + L.start, wnd ? wnd + L.start : nullptr, L.n, c->K, window, c->has_v, la,
+                                         L.act, L.row_off, L.step1, L.act1, L.step1e, L.idx1, c->acc_len + L.start,
+                                         L.counters);
   c->launches++;
 }
 
@@ -238,6 +264,9 @@ struct DraftArgs {
   const float* y;
   const float* v;
   const int* v_off;  // device: first row of v for this lane, or null
+  const int* idx1;     // look-ahead: row of v per active position, -1 = take vsave[chain]
+  const float* vsave;  // look-ahead: v_a saved by the previous round, by chain position
+  int la;
   Tables tab;
   float* Yhat;
   int* row_step;
@@ -276,21 +305,24 @@ __device__ __forceinline__ void draft_store(const DraftArgs& A, int row, int a, 
 }
 
 __global__ void __launch_bounds__(kDraftThreads) draft_kernel(const DraftArgs A) {
-  __shared__ float4 s_pt[kMaxWindow - 1][kDraftQ];  // noise, then drafted points, per slot (parallel form)
+  __shared__ float4 s_pt[kMaxWindow][kDraftQ];  // noise, then drafted points, per slot (parallel form)
   const int p = blockIdx.x;
   if (p >= A.cnt->n_active) return;
   const int j = A.act[p];
   const int a = A.a[j];
   const int w = chain_window(A.wnd, j, A.window, A.K, a);
   const int row0 = A.row_off[p];
+  const int nr = drafted_rows(w, a, A.K, A.la);  // slots 1..nr are drafted
+  const float* vrow = (A.la && A.idx1[p] < 0) ? A.vsave + (size_t)j * A.d
+                                               : A.v + (size_t)((A.la ? A.idx1[p] : (A.v_off ? *A.v_off : 0) + p)) * A.d;
   const uint32_t chain = (uint32_t)(A.chain_base + (uint64_t)j);
   if (!A.par) {
     // large batches: one thread owns 4 dims and walks the window; nothing is staged
     const int q = blockIdx.y * kDraftThreads + threadIdx.x;
     if (q < A.nq) {
       float4 yh = load4(A.y + (size_t)j * A.d, q, A.d, A.vec);
-      const float4 v = load4(A.v + (size_t)((A.v_off ? *A.v_off : 0) + p) * A.d, q, A.d, A.vec);
-      for (int k = 1; k < w; ++k) {
+      const float4 v = load4(vrow, q, A.d, A.vec);
+      for (int k = 1; k <= nr; ++k) {
         const int i = a + k - 1;  // step i -> i+1 uses eta_i, sigma_{i+1}, xi_{i+1}
         const float eta = A.tab.eta[i], sig = A.tab.sig[i];
         const float4 xi = xi4((uint32_t)q, (uint32_t)(i + 1), chain, A.keys);
@@ -308,12 +340,12 @@ __global__ void __launch_bounds__(kDraftThreads) draft_kernel(const DraftArgs A)
     const int q = blockIdx.y * kDraftQ + ql;
     const bool q_ok = q < A.nq;
     if (q_ok)
-      for (int k = 1 + ks; k < w; k += kSlotLanes) s_pt[k - 1][ql] = xi4((uint32_t)q, (uint32_t)(a + k), chain, A.keys);
+      for (int k = 1 + ks; k <= nr; k += kSlotLanes) s_pt[k - 1][ql] = xi4((uint32_t)q, (uint32_t)(a + k), chain, A.keys);
     __syncthreads();
     if (ks == 0 && q_ok) {
       float4 yh = load4(A.y + (size_t)j * A.d, q, A.d, A.vec);
-      const float4 v = load4(A.v + (size_t)((A.v_off ? *A.v_off : 0) + p) * A.d, q, A.d, A.vec);
-      for (int k = 1; k < w; ++k) {
+      const float4 v = load4(vrow, q, A.d, A.vec);
+      for (int k = 1; k <= nr; ++k) {
         const int i = a + k - 1;
         const float eta = A.tab.eta[i], sig = A.tab.sig[i];
         const float4 xi = s_pt[k - 1][ql];
@@ -326,10 +358,10 @@ __global__ void __launch_bounds__(kDraftThreads) draft_kernel(const DraftArgs A)
     }
     __syncthreads();
     if (q_ok)
-      for (int k = 1 + ks; k < w; k += kSlotLanes) draft_store(A, row0 + k - 1, a, k, q, s_pt[k - 1][ql]);
+      for (int k = 1 + ks; k <= nr; k += kSlotLanes) draft_store(A, row0 + k - 1, a, k, q, s_pt[k - 1][ql]);
   }
   // row maps, conditioning, time embedding and zero padding: the chain's blocks share the slots
-  for (int k = 1 + (int)blockIdx.y; k < w; k += gridDim.y) {
+  for (int k = 1 + (int)blockIdx.y; k <= nr; k += gridDim.y) {
     const int row = row0 + k - 1;
     if (threadIdx.x == 0) {
       A.row_step[row] = a + k;
@@ -351,7 +383,8 @@ __global__ void __launch_bounds__(kDraftThreads) draft_kernel(const DraftArgs A)
 }
 
 void launch_draft(Ctx* c, const Lane& L, int window, const float* v_base, const int* v_off_dev) {
-  if (window <= 1 || L.n == 0) return;
+  const bool la = c->lookahead && L.idx1;  // look-ahead drafts a row even for a window of one step
+  if ((window <= 1 && !la) || L.n == 0) return;
   const int* wnd = round_windows(c, window);
   DraftArgs A{};
   A.d = c->d;
@@ -369,6 +402,9 @@ void launch_draft(Ctx* c, const Lane& L, int window, const float* v_base, const 
   A.y = c->y + (size_t)L.start * c->d;
   A.v = v_base;
   A.v_off = v_off_dev;
+  A.la = la ? 1 : 0;
+  A.idx1 = L.idx1;
+  A.vsave = c->vsave;
   A.tab = c->tab;
   A.Yhat = c->Yhat;
   A.row_step = c->row_step;
@@ -420,6 +456,10 @@ struct VerifyArgs {
   float* y;
   const float* v;
   const int* v_off;  // device: first row of v for this lane, or null
+  const int* idx1;   // look-ahead: row of v per active position, -1 = take vsave[chain]
+  float* vsave;      // look-ahead: where a fully accepted window leaves v_a of the next round
+  int* has_v;
+  int la;
   const float* Yhat;
   const float* G;
   Tables tab;
@@ -441,7 +481,8 @@ __global__ void __launch_bounds__(256) verify_kernel(const VerifyArgs A) {
   const int row0 = A.row_off[p];
   const uint32_t chain = (uint32_t)(A.chain_base + (uint64_t)j);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
-  const float* vrow = A.v + (size_t)((A.v_off ? *A.v_off : 0) + p) * A.d;
+  const float* vrow = (A.la && A.idx1[p] < 0) ? A.vsave + (size_t)j * A.d
+                                               : A.v + (size_t)((A.la ? A.idx1[p] : (A.v_off ? *A.v_off : 0) + p)) * A.d;
   const float nan = __int_as_float(0x7fc00000);
 
   // ln u of every slot (one Philox call each), and the diagnostics of slot 1: proposal mean == target
@@ -571,6 +612,18 @@ __global__ void __launch_bounds__(256) verify_kernel(const VerifyArgs A) {
       store4(yrow, q, A.d, A.vec, o);
     }
   }
+  if (A.la) {
+    // look-ahead: after a fully accepted window the drift at its last drafted point, evaluated in this
+    // round's batched pass, is v_a of the next round (Algorithm 1's first model call at y_{a+w})
+    const bool reuse = (n == w) && (a + w < A.K);
+    __syncthreads();  // vrow may be this chain's saved row: every thread is done with it
+    if (reuse) {
+      const float* glast = A.G + (size_t)(row0 + w - 1) * A.d;
+      float* dst = A.vsave + (size_t)j * A.d;
+      for (int q = tid; q < A.nq; q += blockDim.x) store4(dst, q, A.d, A.vec, load4(glast, q, A.d, A.vec));
+    }
+    if (tid == 0) A.has_v[j] = reuse ? 1 : 0;
+  }
   if (tid == 0) {
     const int adv = (n < w) ? n + 1 : w;
     A.a[j] = a + adv;
@@ -613,6 +666,10 @@ void launch_verify(Ctx* c, const Lane& L, int window, bool use_u, const float* G
   A.y = c->y + (size_t)L.start * c->d;
   A.v = v_base;
   A.v_off = v_off_dev;
+  A.la = (c->lookahead && L.idx1) ? 1 : 0;
+  A.idx1 = L.idx1;
+  A.vsave = c->vsave;
+  A.has_v = c->has_v;
   A.Yhat = c->Yhat;
   A.G = G;
   A.tab = c->tab;

@@ -61,7 +61,7 @@ def rel_l2(a, b):
 
 
 def lockstep(sampler, wl, n_chains, n_rounds, chain_base=0, check_chains=None, cond=None, log=None,
-             cascade=False, all_slots=False, adaptive=False, sigma2=None, y0=None):
+             cascade=False, all_slots=False, adaptive=False, sigma2=None, y0=None, lookahead=False):
     """Runs `n_rounds` rounds on the GPU; before each round the oracle is restarted from the
     GPU's state and must reproduce ln u, ln ratio, the accepted prefix and the new state."""
     g = oden.from_workload(wl)
@@ -70,6 +70,7 @@ def lockstep(sampler, wl, n_chains, n_rounds, chain_base=0, check_chains=None, c
     check = list(range(n_chains)) if check_chains is None else list(check_chains)
     sampler.reset(n_chains, chain_base, cond=cond, y0=y0)
     worst = dict(y=0.0, lr=0.0, lr_over_tol=0.0, lu=0.0, exempt=0, decided=0, rounds=0, slots=0)
+    saved = np.zeros(n_chains, dtype=bool)   # look-ahead: chains whose last round accepted its whole window
     for r in range(n_rounds):
         a0, y0, _ = [t.cpu().numpy() for t in sampler.get_state()]
         if adaptive:      # every chain has its own speculation length this round
@@ -84,7 +85,16 @@ def lockstep(sampler, wl, n_chains, n_rounds, chain_base=0, check_chains=None, c
         assert st.n_active_before == int(np.sum(a0 < wl.K))
         assert st.n_active_after == int(np.sum(a1 < wl.K))
         assert st.accepted_total == int(np.sum(a1 - a0))
-        assert st.rows_pass2 == int(np.sum(np.minimum(theta, wl.K - a0)[a0 < wl.K] - 1))
+        w_all = np.minimum(theta, wl.K - a0)
+        if lookahead:
+            # one more drafted row wherever a step lies beyond the window; the first model call only for
+            # the chains that did not accept their whole window in the previous round
+            assert st.rows_pass2 == int(np.sum((w_all - 1 + (a0 + w_all < wl.K))[a0 < wl.K]))
+            assert st.rows_pass1 == int(np.sum((a0 < wl.K) & ~saved))
+            saved = (a0 < wl.K) & (acc == w_all) & (a0 + w_all < wl.K)
+        else:
+            assert st.rows_pass2 == int(np.sum(w_all[a0 < wl.K] - 1))
+            assert st.rows_pass1 == st.n_active_before
         worst["rounds"] += 1
         for j in check:
             if a0[j] >= wl.K:

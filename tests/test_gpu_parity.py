@@ -193,6 +193,77 @@ def test_adaptive_window_whole_run_and_invariance():
     assert compared >= 3
 
 
+@pytest.mark.parametrize("adaptive", [False, True])
+@pytest.mark.parametrize("name,chains,rounds", [("cfg1_gmm2d", 16, 40), ("gmm_odd", 9, 30), ("cfg2_gauss64", 24, 12),
+                                                ("mlp_tiny", 5, 25), ("mlp_ragged", 37, 8), ("cfg3_policy", 64, 3)])
+def test_lockstep_lookahead(name, chains, rounds, adaptive):
+    """ASD_FLAG_LOOKAHEAD: the batched pass also evaluates the drift at the end of each window, and a
+    chain that accepted its whole window skips the first model call of its next round.  Every round is
+    still the oracle's round from the same state (the saved drift is the drift at that state), and the
+    row counts of both passes follow the rule."""
+    from paper_2505_03983_b200.binding import FLAG_ADAPTIVE_WINDOW, FLAG_LOOKAHEAD
+    wl = workloads.make(name, chains=chains)
+    with _sampler(wl, flags=FLAG_LOOKAHEAD | (FLAG_ADAPTIVE_WINDOW if adaptive else 0)) as s:
+        worst = lockstep(s, wl, chains, rounds, chain_base=700, cond=wl.cond if wl.kind == "mlp" and wl.d_cond else None,
+                         log=_log, adaptive=adaptive, lookahead=True)
+    assert worst["decided"] > 0
+
+
+@pytest.mark.parametrize("name,chains,K", [("cfg1_gmm2d", 33, None), ("cfg2_gauss64", 16, 300), ("gmm_wide", 3, None)])
+def test_lookahead_whole_run_equals_default(name, chains, K):
+    """The analytic drifts are computed row by row, so moving an evaluation into the previous round's
+    batch changes no bit: whole runs with and without look-ahead give the same samples in the same number
+    of rounds with fewer sequential model calls, and so does the sequential sampler."""
+    from paper_2505_03983_b200.binding import FLAG_LOOKAHEAD
+    wl = workloads.make(name, chains=chains) if K is None else workloads.make(name, chains=chains, K=K)
+    with _sampler(wl) as s0:
+        s0.reset(chains, 11)
+        y0, r0, st0 = s0.sample()
+        s0.reset(chains, 11)
+        q0, _ = s0.sequential_ddpm()
+    with _sampler(wl, flags=FLAG_LOOKAHEAD) as s1:
+        s1.reset(chains, 11)
+        y1, r1, st1 = s1.sample()
+        s1.reset(chains, 11)
+        q1, sq = s1.sequential_ddpm()
+        # a restart after a partial run must not reuse a stale drift
+        s1.reset(chains, 11)
+        for _ in range(3):
+            s1.round(want_stats=False)
+        s1.reset(chains, 11)
+        y2, r2, _ = s1.sample()
+    assert torch.equal(y0, y1) and torch.equal(r0, r1)
+    assert torch.equal(y0, y2) and torch.equal(r0, r2)
+    assert torch.equal(q0, q1)
+    assert sq.rows_total == chains * wl.K          # one drift evaluation per step, as without the flag
+    _log(f"look-ahead {name}: drift rows {st0.rows_total} -> {st1.rows_total}, rounds mean {r0.float().mean():.1f}")
+
+
+def test_lookahead_network_whole_run():
+    """Network denoiser: the saved drift comes out of a different GEMM batch, so whole runs agree with the
+    oracle's (not bit for bit with the default mode) on chains whose every decision is well outside the
+    ln-ratio tolerance of the bf16 network."""
+    from paper_2505_03983_b200.binding import FLAG_LOOKAHEAD
+    wl = workloads.make("mlp_tiny", chains=24)
+    with _sampler(wl, flags=FLAG_LOOKAHEAD) as s:
+        s.reset(24, 0, cond=wl.cond)
+        y, rounds, st = s.sample()
+    with _sampler(wl) as s0:
+        s0.reset(24, 0, cond=wl.cond)
+        _, _, st0 = s0.sample()
+    ref = oracle_run(wl, range(24))
+    y, rounds = y.cpu().numpy(), rounds.cpu().numpy()
+    tol_y, _ = tolerances(wl.kind)
+    compared = 0
+    for j, res in enumerate(ref):
+        if res.min_margin > 1e-2:
+            compared += 1
+            assert rounds[j] == res.rounds, (j, rounds[j], res.rounds)
+            assert rel_l2(y[j].astype(np.float64), res.y) < tol_y
+    _log(f"look-ahead mlp_tiny: compared {compared} of 24, drift rows {st0.rows_total} -> {st.rows_total}")
+    assert compared >= 10
+
+
 @pytest.mark.parametrize("mapping,pred", [("sl", "eps"), ("ancestral", "eps"), ("ancestral", "v")])
 def test_ddpm_front_end_chain(mapping, pred):
     """A chain built by asd_ddpm_schedule (non-uniform steps, explicit variances in the ancestral
