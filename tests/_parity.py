@@ -61,9 +61,12 @@ def rel_l2(a, b):
 
 
 def lockstep(sampler, wl, n_chains, n_rounds, chain_base=0, check_chains=None, cond=None, log=None,
-             cascade=False, all_slots=False, adaptive=False, sigma2=None, y0=None, lookahead=False):
+             cascade=False, all_slots=False, adaptive=False, sigma2=None, y0=None, lookahead=False,
+             check_rounds=None):
     """Runs `n_rounds` rounds on the GPU; before each round the oracle is restarted from the
-    GPU's state and must reproduce ln u, ln ratio, the accepted prefix and the new state."""
+    GPU's state and must reproduce ln u, ln ratio, the accepted prefix and the new state.
+    check_rounds(r, stats) -> bool picks the rounds the oracle re-runs (default: all); the counters are
+    checked in every round."""
     g = oden.from_workload(wl)
     sch = oasd.make_schedule(wl.t, sigma2)
     tol_y, tol_r = tolerances(wl.kind)
@@ -95,6 +98,8 @@ def lockstep(sampler, wl, n_chains, n_rounds, chain_base=0, check_chains=None, c
         else:
             assert st.rows_pass2 == int(np.sum(w_all[a0 < wl.K] - 1))
             assert st.rows_pass1 == st.n_active_before
+        if check_rounds is not None and not check_rounds(r, st):
+            continue
         worst["rounds"] += 1
         for j in check:
             if a0[j] >= wl.K:

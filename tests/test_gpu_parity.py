@@ -119,6 +119,18 @@ def test_lockstep_full_size_configs_sampled_chains(name, check, rounds, cascade)
     assert worst["decided"] > 0
 
 
+def test_lockstep_cfg4_whole_run_sampled_rounds():
+    """cfg4 to the end of the run: every 25th round and the round in which the last chain finishes, on
+    four chains (the first rounds of all sampled chains are covered above)."""
+    wl = workloads.make("cfg4_image")
+    with _sampler(wl) as s:
+        worst = lockstep(s, wl, wl.chains, 10 ** 6, check_chains=[0, 7, 13, 31], log=_log, cascade=True,
+                         check_rounds=lambda r, st: r % 25 == 24 or st.n_active_after == 0)
+        a, _, rounds = [t.cpu().numpy() for t in s.get_state()]
+    assert np.all(a == wl.K) and worst["rounds"] >= 5 and worst["decided"] > 0
+    assert math.ceil(wl.K / wl.window) <= rounds.min() and rounds.max() <= math.ceil(wl.K / 2)
+
+
 def test_lockstep_bench_workload_sampled_chains():
     """The bench's own launch configuration (cfg-4 network, 512 chains x window 64: 32256 drafted rows
     per round) for two rounds; the oracle re-runs a sample of the chains from the GPU's state."""
@@ -130,7 +142,7 @@ def test_lockstep_bench_workload_sampled_chains():
 # ------------------------------------------------------------------ lock-step rounds
 @pytest.mark.parametrize("all_slots", [False, True])
 @pytest.mark.parametrize("name,chains,rounds", [
-    ("cfg1_gmm2d", 16, 60), ("gmm_odd", 9, 30), ("gmm_wide", 3, 6), ("gauss_small", 11, 40), ("cfg2_gauss64", 24, 12),
+    ("cfg1_gmm2d", 16, 60), ("gmm_odd", 9, 30), ("gmm_wide", 3, 6), ("gmm_max_d", 2, 4), ("gauss_small", 11, 40), ("cfg2_gauss64", 24, 12),
     ("mlp_tiny", 5, 25), ("mlp_odd", 7, 12), ("mlp_ragged", 37, 8), ("cfg3_policy", 64, 3)])
 def test_lockstep_rounds(name, chains, rounds, all_slots):
     """all_slots=False is the production path (the verify kernel stops at the first rejected slot);

@@ -172,6 +172,9 @@ def make(name: str, *, chains: Optional[int] = None, K: Optional[int] = None,
     if name == "gmm_wide":
         # a wide, odd dimension: many float4 groups per row and a ragged tail in every kernel
         return _gmm(name, 4099, 3, 0.5, ov(K, 12), ov(window, 6), ov(chains, 3), s, box=0.05)
+    if name == "gmm_max_d":
+        # the largest dimension the library accepts
+        return _gmm(name, 65536, 2, 0.5, ov(K, 6), ov(window, 4), ov(chains, 2), s, box=0.02)
     if name == "gmm_odd":
         return _gmm(name, 5, 3, 0.5, ov(K, 50), ov(window, 7), ov(chains, 9), s)
     if name == "gauss_small":
