@@ -309,8 +309,8 @@ __device__ __forceinline__ void epilogue_chunk(const GemmArgs& g, int row, int c
 }
 
 // What the fused tail of a layer reads from global memory for 32 columns of one row: the residual
-// h_{l-1} (32 bf16) for EPI_HID, the state y (32 fp32) for EPI_OUT, nothing for EPI_IN.  Fetched one
-// chunk ahead of the arithmetic so that its latency overlaps the previous chunk.
+// h_{l-1} (32 bf16) for EPI_HID, the state y (32 fp32) for EPI_OUT, nothing for EPI_IN.  Fetched a few
+// chunks ahead of the arithmetic (kEpiAhead) so that its latency overlaps the chunks before it.
 template <int EPI>
 struct EpiOperand {
   uint4 v[EPI == EPI_OUT ? 8 : (EPI == EPI_HID ? 4 : 1)];
@@ -375,6 +375,11 @@ __device__ __forceinline__ void epi_apply(const GemmArgs& g, int row, int col0, 
   }
 }
 
+// How many 32-column chunks ahead the operand is fetched: one L2 round trip under load is longer than the
+// arithmetic of one chunk (16 registers per chunk for the residual, 32 for the state).
+template <int EPI>
+constexpr int kEpiAhead = (EPI == EPI_OUT) ? 2 : 3;
+
 // Epilogue of one accumulator tile row: this thread owns output row `row` (tensor-memory lane) and walks
 // its BN columns in chunks of 32.  tcgen05.ld is warp-collective, so every lane runs the loop and only
 // the global accesses are predicated on row_ok.
@@ -384,15 +389,18 @@ __device__ __forceinline__ void epilogue_tile(const GemmArgs& g, uint32_t taddr0
   const bool full_vec =
       (n0 + BN <= g.n_out) && (EPI == EPI_OUT ? (g.n_out % 4 == 0) : (g.ld_h % 8 == 0));  // warp-uniform
   if (full_vec) {
-    EpiOperand<EPI> op[2];
-    if (row_ok) epi_fetch<EPI>(op[0], g, row, n0, ysrc_row);
+    constexpr int D = kEpiAhead<EPI>;  // chunks whose operand is in flight ahead of the arithmetic
+    EpiOperand<EPI> op[D + 1];
+#pragma unroll
+    for (int i = 0; i < D; ++i)
+      if (i < BN / 32 && row_ok) epi_fetch<EPI>(op[i], g, row, n0 + i * 32, ysrc_row);
 #pragma unroll
     for (int c = 0; c < BN / 32; ++c) {
       uint32_t r[32];
       tc_ld32(taddr0 + (uint32_t)(c * 32), r);
-      if (c + 1 < BN / 32 && row_ok) epi_fetch<EPI>(op[(c + 1) & 1], g, row, n0 + (c + 1) * 32, ysrc_row);
+      if (c + D < BN / 32 && row_ok) epi_fetch<EPI>(op[(c + D) % (D + 1)], g, row, n0 + (c + D) * 32, ysrc_row);
       tc_wait_ld();
-      if (row_ok) epi_apply<EPI>(g, row, n0 + c * 32, r, op[c & 1], cs, co);
+      if (row_ok) epi_apply<EPI>(g, row, n0 + c * 32, r, op[c % (D + 1)], cs, co);
     }
   } else {
 #pragma unroll 1
