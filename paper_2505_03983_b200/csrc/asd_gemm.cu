@@ -30,6 +30,8 @@ constexpr int BM = 128;       // rows of an output tile = MMA M = tensor-memory 
 constexpr int BK = 64;        // bf16 elements per k-block = one 128-byte swizzle row
 constexpr int UMMA_K = 16;    // k extent of one tcgen05.mma (bf16)
 constexpr int kGemmThreads = 192;
+constexpr int kPairEpiWarps = 8;  // CTA-pair kernel: two epilogue warps per tensor-memory lane quarter, half the columns each
+constexpr int kPairThreads = 64 + 32 * kPairEpiWarps;
 constexpr int kEpiWarp0 = 2;  // warps 2..5 are epilogue warps
 constexpr long long kWaitCycles = 400000000ll;  // ~0.2 s at 1.9 GHz per wait
 
@@ -574,7 +576,7 @@ struct PairCfg {
 };
 
 template <int BN, int EPI>
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemmThreads, 1)
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPairThreads, 1)
 gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_w,
                  const GemmArgs g) {
   using C = PairCfg<BN>;
@@ -610,7 +612,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
     }
     for (int b = 0; b < 2; ++b) {
       mbar_init(accf_bar(b), 1);
-      mbar_init(acce_bar(b), 8);
+      mbar_init(acce_bar(b), 2 * kPairEpiWarps);  // every epilogue warp of both CTAs
     }
     *dead = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -706,8 +708,10 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
         co = g.c_out[step];
         ysrc_row = g.ysrc + (size_t)(g.row_map ? g.row_map[row] : row) * g.n_out;
       }
-      epilogue_tile<EPI, BN>(g, tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN), row, row_ok, n0, cs,
-                             co, ysrc_row);
+      constexpr int kCols = BN / (kPairEpiWarps / 4);  // this warp's share of the tile's columns
+      const int part = (warp - kEpiWarp0) >> 2;
+      epilogue_tile<EPI, kCols>(g, tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN + part * kCols), row,
+                                row_ok, n0 + part * kCols, cs, co, ysrc_row);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive_cluster(map_to_cta(acce_bar(acc), 0));
@@ -1043,7 +1047,7 @@ asd_status launch_gemm_pair_t(Ctx* c, const void* a_ptr, int a_cols, const void*
   }
   const int tiles = ((m_bound + 2 * BM - 1) / (2 * BM)) * ((g.n_out + BN - 1) / BN);
   const int pairs = std::max(1, std::min(tiles, c->num_sms / 2));
-  gemm_pair_kernel<BN, EPI><<<2 * pairs, kGemmThreads, C::kSmemBytes, c->stream>>>(ma, mw, g);
+  gemm_pair_kernel<BN, EPI><<<2 * pairs, kPairThreads, C::kSmemBytes, c->stream>>>(ma, mw, g);
   c->launches++;
   return ASD_OK;
 }
