@@ -1,7 +1,7 @@
 // The network denoiser's forward pass as a chain of bf16 x bf16 -> fp32 GEMMs on the 5th-generation
 // tensor cores: operands staged in shared memory by TMA (128-byte swizzle), tcgen05.mma issued by one
 // thread with the accumulator in tensor memory, a warp-specialised persistent kernel (one TMA warp,
-// one MMA warp, four epilogue warps) with a multi-stage mbarrier pipeline and a double-buffered
+// one MMA warp, four or eight epilogue warps) with a multi-stage mbarrier pipeline and a double-buffered
 // accumulator so that the epilogue of one tile overlaps the MMAs of the next.
 //
 //   Y[m, n] = sum_k A[m, k] W[n, k]      A: activations [rows, K] row-major, W: weights [N, K] row-major
@@ -32,6 +32,8 @@ constexpr int UMMA_K = 16;    // k extent of one tcgen05.mma (bf16)
 constexpr int kGemmThreads = 192;
 constexpr int kPairEpiWarps = 8;  // CTA-pair kernel: two epilogue warps per tensor-memory lane quarter, half the columns each
 constexpr int kPairThreads = 64 + 32 * kPairEpiWarps;
+constexpr int kSkinnyThreads = 64 + 32 * 8;  // weight-streaming kernel: four epilogue warps, or (more than 32 rows) eight:
+                                             // two per lane quarter, alternate rows each
 constexpr int kEpiWarp0 = 2;  // warps 2..5 are epilogue warps
 constexpr long long kWaitCycles = 400000000ll;  // ~0.2 s at 1.9 GHz per wait
 
@@ -563,9 +565,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
 // Each CTA stages only its own 128 rows of A and BN/2 of the tile's BN weight rows (for BN = 256: 32 KB
 // per k-block instead of 48 KB for the same 128 x 256 x 64 of tensor work per SM), so the L2 -> shared-memory
 // stream per flop drops by a third.  Rank 0 of the pair issues the MMAs; both
-// CTAs run a TMA warp and four epilogue warps on their own 128 accumulator rows.
+// CTAs run a TMA warp and eight epilogue warps (two per lane quarter) on their own 128 accumulator rows.
 //   full[s]   in rank 0, completed by both CTAs' TMA bytes          empty[s]  in each CTA, MMA commit
-//   accf[b]   in each CTA, MMA commit                               acce[b]   in rank 0, 8 epilogue warps
+//   accf[b]   in each CTA, MMA commit                               acce[b]   in rank 0, all 16 epilogue warps
 // ---------------------------------------------------------------------------------------------------
 template <int BN>
 struct PairCfg {
@@ -750,7 +752,7 @@ constexpr int kSkinnyMaxRows = 256;    // one row block: at 512 rows the CTA-pai
 __host__ __device__ constexpr int skinny_stage_bytes(int m_pad) { return (BM + m_pad) * BK * 2; }
 
 template <int EPI>
-__global__ void __cluster_dims__(kSplit, 1, 1) __launch_bounds__(kGemmThreads, 1)
+__global__ void __cluster_dims__(kSplit, 1, 1) __launch_bounds__(kSkinnyThreads, 1)
 gemm_skinny_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x,
                    const GemmArgs g, const int m_pad, const int S) {
   extern __shared__ uint8_t smem_raw[];
@@ -876,7 +878,9 @@ gemm_skinny_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
     mbar_wait(accf_bar, 0u, dead, g.err);
     tc_fence_after();
     float* part = reinterpret_cast<float*>(tiles_ptr);  // the stage buffers are idle now: [m_pad][128] fp32
-    for (int c0 = 0; c0 < m_pad; c0 += 16) {
+    const int halves = ((int)(blockDim.x >> 5) - kEpiWarp0) >> 2;  // epilogue warps per lane quarter: 1 or 2
+    const int half = (warp - kEpiWarp0) >> 2;  // they take alternate groups of 16 rows
+    for (int c0 = half * 16; c0 < m_pad; c0 += 16 * halves) {
       uint32_t r[16];
       if (kb1 > kb0) {
         tc_ld16(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)c0, r);
@@ -910,11 +914,13 @@ gemm_skinny_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
       // distributed shared memory, residual / state and per-row scalars from global memory) are issued
       // before the first store, so one memory latency is paid per group instead of per row
       constexpr int R = 8;
-      for (int lr0 = (int)rank; lr0 < m; lr0 += R * kSplit) {
+      const int kRowStep = kSplit * (((int)(blockDim.x >> 5) - kEpiWarp0) >> 2);  // this warp's rows: every kRowStep-th
+      const int half = (warp - kEpiWarp0) >> 2;
+      for (int lr0 = (int)rank + half * kSplit; lr0 < m; lr0 += R * kRowStep) {
         float acc[R], opnd[R], cs[R], co[R];
 #pragma unroll
         for (int u = 0; u < R; ++u) {
-          const int lr = min(lr0 + u * kSplit, m - 1);  // clamped rows are loaded but not stored
+          const int lr = min(lr0 + u * kRowStep, m - 1);  // clamped rows are loaded but not stored
           const int row = row0 + lr;
           float a = 0.f;
 #pragma unroll
@@ -931,7 +937,7 @@ gemm_skinny_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
         }
 #pragma unroll
         for (int u = 0; u < R; ++u) {
-          const int lr = lr0 + u * kSplit;
+          const int lr = lr0 + u * kRowStep;
           if (lr < m) {
             const int row = row0 + lr;
             float x = acc[u] + bias;
@@ -1075,7 +1081,7 @@ asd_status launch_gemm_skinny(Ctx* c, const void* a_ptr, int a_cols, const void*
   // anything that kernel wrote.
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = grid;
-  cfg.blockDim = dim3(kGemmThreads);
+  cfg.blockDim = dim3(m_pad > 32 ? kSkinnyThreads : kGemmThreads);  // a second set of epilogue warps pays from 33 rows
   cfg.dynamicSmemBytes = (size_t)smem;
   cfg.stream = c->stream;
   cudaLaunchAttribute attr[1];
