@@ -599,11 +599,13 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = cluster_ctarank();
   const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
-  const int m = min(*g.m_dev, g.m_cap);
-  const int tiles_m = (m + 2 * BM - 1) / (2 * BM);
   const int tiles_n = (g.n_out + BN - 1) / BN;
-  const int n_tiles = tiles_m * tiles_n;
   const int num_kb = (g.k_dim + BK - 1) / BK;
+
+  // Programmatic dependent launch: the next kernel of the stream may be scheduled from now on (its CTAs start as
+  // SMs become free), and this kernel sets up its barriers and tensor memory while the previous one finishes;
+  // everything that kernel wrote (the row count included) is read after grid_dependency_wait() below.
+  grid_launch_dependents();
 
   if (threadIdx.x == 0) {
     prefetch_tmap(&map_a);
@@ -631,6 +633,10 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
   cluster_sync_all();  // the peer's barriers are initialised before anything arrives on them
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  grid_dependency_wait();
+  const int m = min(*g.m_dev, g.m_cap);
+  const int tiles_m = (m + 2 * BM - 1) / (2 * BM);
+  const int n_tiles = tiles_m * tiles_n;
 
   if (warp == 0) {
     // ---------------- TMA producer (both CTAs) ----------------
@@ -1053,7 +1059,20 @@ asd_status launch_gemm_pair_t(Ctx* c, const void* a_ptr, int a_cols, const void*
   }
   const int tiles = ((m_bound + 2 * BM - 1) / (2 * BM)) * ((g.n_out + BN - 1) / BN);
   const int pairs = std::max(1, std::min(tiles, c->num_sms / 2));
-  gemm_pair_kernel<BN, EPI><<<2 * pairs, kPairThreads, C::kSmemBytes, c->stream>>>(ma, mw, g);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(2 * pairs);
+  cfg.blockDim = dim3(kPairThreads);
+  cfg.dynamicSmemBytes = (size_t)C::kSmemBytes;
+  cfg.stream = c->stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  if (cudaLaunchKernelEx(&cfg, gemm_pair_kernel<BN, EPI>, ma, mw, g) != cudaSuccess) {
+    c->err = std::string("pair GEMM launch failed: ") + cudaGetErrorString(cudaGetLastError());
+    return ASD_ERR_CUDA;
+  }
   c->launches++;
   return ASD_OK;
 }
