@@ -33,7 +33,7 @@ DEFAULT_WORKLOAD = "sweep_b512_w64"   # cfg-4 denoiser, 512 chains x window 64, 
 # dram__bytes_read.sum + dram__bytes_write.sum of one pass-2 hidden-layer launch of gemm_pair_kernel<256, EPI_HID>
 # at full row count, from the ncu capture summarised in profiles/gemm_pair_hidden_sweep_b512_w16.md; set an entry to
 # None when that kernel changes until the counters are taken again
-NCU_TRAFFIC_BYTES_PER_LAUNCH = {"sweep_b512_w64": 401_028_864 + 245_600_256}
+NCU_TRAFFIC_BYTES_PER_LAUNCH = {"sweep_b512_w64": 391_901_184 + 244_783_872}
 METRIC = "samples_per_sec"
 UNIT = "samples/s"
 
