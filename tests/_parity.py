@@ -144,7 +144,7 @@ def lockstep(sampler, wl, n_chains, n_rounds, chain_base=0, check_chains=None, c
                 if a0[j] >= wl.K:
                     assert theta1[j] == theta[j] and ema81[j] == ema8[j]
                     continue
-                pol = oasd.AdaptiveWindow(sampler.window, int(ema8[j]))
+                pol = oasd.AdaptiveWindow(min(sampler.window, wl.K), int(ema8[j]))   # a window beyond K acts like K
                 pol.update(int(a1[j] - a0[j]))
                 assert (ema81[j], theta1[j]) == (pol.ema8, pol.theta()), (r, j)
     if log is not None:

@@ -251,6 +251,26 @@ def test_lookahead_whole_run_equals_default(name, chains, K):
     _log(f"look-ahead {name}: drift rows {st0.rows_total} -> {st1.rows_total}, rounds mean {r0.float().mean():.1f}")
 
 
+@pytest.mark.parametrize("K,window,chains", [(1, 1, 3), (2, 2, 1), (5, 8, 2), (7, 3, 4)])
+def test_lookahead_short_chains(K, window, chains):
+    """Look-ahead at the ends of its range: a single step (nothing to look ahead to), windows that reach or pass
+    the last step (no extra row is drafted there), one chain; with adaptive windows on top."""
+    from paper_2505_03983_b200.binding import FLAG_ADAPTIVE_WINDOW, FLAG_LOOKAHEAD
+    for name in ("cfg1_gmm2d", "mlp_tiny"):
+        wl = workloads.make(name, K=K, window=window, chains=chains)
+        cond = wl.cond if wl.kind == "mlp" and wl.d_cond else None
+        # (per-chain windows range over 2..window: nothing to adapt for a window of one step)
+        for flags in (FLAG_LOOKAHEAD,) + ((FLAG_LOOKAHEAD | FLAG_ADAPTIVE_WINDOW,) if window >= 2 else ()):
+            with _sampler(wl, flags=flags) as s:
+                lockstep(s, wl, chains, K + 1, chain_base=3, cond=cond, log=None,
+                         adaptive=bool(flags & FLAG_ADAPTIVE_WINDOW), lookahead=True)
+                a, _, rounds = [t.cpu().numpy() for t in s.get_state()]
+                assert np.all(a == K) and np.all(rounds >= 1)
+                s.reset(chains, 3, cond=cond)
+                y, r, _ = s.sample()
+                assert torch.isfinite(y).all() and torch.all(r >= math.ceil(K / max(window, 2)) if K > 1 else r == 1)
+
+
 def test_lookahead_network_whole_run():
     """Network denoiser: the saved drift comes out of a different GEMM batch, so whole runs agree with the
     oracle's (not bit for bit with the default mode) on chains whose every decision is well outside the
