@@ -79,6 +79,16 @@ class ClockSampler:
             self.proc.kill()
         sm, mx, reasons = [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        late = False
+        if not self.rows:
+            # a timed region shorter than nvidia-smi's first report: one query right after it instead
+            try:
+                out = subprocess.run(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
+                                      "--format=csv,noheader,nounits"], capture_output=True, text=True, timeout=10).stdout
+                self.rows = [[x.strip() for x in line.split(",")] for line in out.splitlines() if line.strip()]
+                late = True
+            except (OSError, subprocess.SubprocessError):
+                pass
         for r in self.rows:
             if len(r) < 6:
                 continue
@@ -89,8 +99,11 @@ class ClockSampler:
             for nm, val in zip(names, r[2:6]):
                 if val.lower().startswith("active"):
                     reasons.add(nm)
-        return dict(sm_mhz=float(np.median(sm)) if sm else None, sm_max_mhz=max(mx) if mx else None,
-                    reasons=sorted(reasons), samples=len(sm))
+        res = dict(sm_mhz=float(np.median(sm)) if sm else None, sm_max_mhz=max(mx) if mx else None,
+                   reasons=sorted(reasons), samples=len(sm))
+        if late:
+            res["note"] = "sampled right after the timed region (it was shorter than the sampling interval)"
+        return res
 
 
 def oracle_sample_rate(wl, budget_s: float, max_rounds: int):
