@@ -361,8 +361,9 @@ __global__ void __launch_bounds__(kDraftThreads) draft_kernel(const DraftArgs A)
       for (int k = 1 + ks; k <= nr; k += kSlotLanes) draft_store(A, row0 + k - 1, a, k, q, s_pt[k - 1][ql]);
   }
   // row maps, conditioning, time embedding and zero padding: the chain's blocks share the slots (this block takes
-  // slots k = 1 + blockIdx.y + i * gridDim.y).  The (slot, element) pairs are walked flat, four per thread at a time
-  // with the loads ahead of the stores, so a thread waits for memory once per four elements, not once per slot.
+  // slots k = 1 + blockIdx.y + i * gridDim.y).  With few blocks in flight (the staged form) the (slot, element) pairs
+  // are walked flat, four per thread at a time with the loads ahead of the stores, so a thread waits for memory once
+  // per four elements, not once per slot.
   const int k_first = 1 + (int)blockIdx.y;
   const int ks = nr >= k_first ? (nr - k_first) / (int)gridDim.y + 1 : 0;
   for (int i = threadIdx.x; i < ks; i += blockDim.x) {
@@ -370,7 +371,21 @@ __global__ void __launch_bounds__(kDraftThreads) draft_kernel(const DraftArgs A)
     A.row_step[row0 + k - 1] = a + k;
     A.row_slot[row0 + k - 1] = j;
   }
-  if (A.X) {
+  if (A.X && !A.par) {
+    // many blocks in flight: slot by slot, no index arithmetic per element
+    const int extra = A.in_pad - A.d;
+    for (int k = k_first; k <= nr; k += gridDim.y) {
+      __nv_bfloat16* xr = A.X + (size_t)(row0 + k - 1) * A.in_pad + A.d;
+      for (int e = threadIdx.x; e < extra; e += blockDim.x) {
+        __nv_bfloat16 val = __float2bfloat16_rn(0.f);
+        if (e < A.d_cond)
+          val = A.cond[(size_t)j * A.d_cond + e];
+        else if (e < A.d_cond + A.d_temb)
+          val = A.temb[(size_t)(a + k) * A.d_temb + (e - A.d_cond)];
+        xr[e] = val;
+      }
+    }
+  } else if (A.X) {
     const int extra = A.in_pad - A.d;
     const int items = ks * extra, stride = (int)blockDim.x;
     const __nv_bfloat16 zero = __float2bfloat16_rn(0.f);
