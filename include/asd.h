@@ -103,7 +103,8 @@ typedef struct {
 typedef struct {
   int32_t d;          /* dimension of y, 1..65536 */
   int32_t K;          /* number of Euler steps, >= 1 */
-  int32_t window;     /* speculation length theta, 1..64 (values > K act like K) */
+  int32_t window;     /* speculation length theta >= 1; values >= K act like K, i.e. theta = infinity:
+                         every round drafts to the end of the grid (workspaces are sized max_chains x window) */
   int32_t max_chains; /* capacity of the batch, >= 1 */
   const double* t;      /* host [K+1], strictly increasing, t[0] >= 0 */
   const double* sigma2; /* host [K]: sigma_{i+1}^2 for the step i -> i+1, or NULL => eta_i
@@ -149,6 +150,21 @@ typedef struct {
  * only the chains whose first call was really made.
  */
 #define ASD_FLAG_LOOKAHEAD 4u
+
+/*
+ * ASD_FLAG_TRAJECTORY: keep Algorithm 1's return value (y_0, ..., y_K) for every chain, not only y_K:
+ * a [max_chains, K + 1, d] float buffer on the device that the verify step fills as chains advance (the
+ * accepted proposal samples, then the resampled state) and asd_get_trajectory copies out.  Row 0 is the
+ * y_0 of asd_reset; after asd_set_state rows below the restored cursor are whatever the context held.
+ */
+#define ASD_FLAG_TRAJECTORY 8u
+
+/*
+ * ASD_FLAG_DEBUG_DUMP: record ln u and ln ratio of the last round per window slot for
+ * asd_debug_last_round (two [max_chains, window] float buffers, written by the verify step every
+ * round).  Implied by ASD_FLAG_DEBUG_ALL_SLOTS.  Without it only the accepted prefix lengths are kept.
+ */
+#define ASD_FLAG_DEBUG_DUMP 16u
 
 typedef struct {
   int32_t n_active_before; /* chains with a < K when the round started */
@@ -240,9 +256,26 @@ asd_status asd_set_window_state(asd_ctx* ctx, const int32_t* window_dev, const i
  * ln u per window slot ([n*window] fp32 each; slots beyond the chain's window are not
  * written; ln ratio of slots after the first rejected one is NaN unless the context was
  * created with ASD_FLAG_DEBUG_ALL_SLOTS) and the accepted prefix length n ([n] int32; -1 for
- * chains that were inactive).  Device buffers, any may be NULL.
+ * chains that were inactive).  Device buffers, any may be NULL.  The two ln arrays need a context
+ * created with ASD_FLAG_DEBUG_DUMP (or ASD_FLAG_DEBUG_ALL_SLOTS): STATE otherwise.
  */
 asd_status asd_debug_last_round(asd_ctx* ctx, float* ln_ratio_dev, float* ln_u_dev, int32_t* accepted_dev);
+
+/*
+ * Algorithm 1's output (y_0, ..., y_K) per chain: traj_dev [n, K + 1, d] fp32 (device).  Rows beyond a
+ * chain's cursor are not yet written.  Needs ASD_FLAG_TRAJECTORY (STATE otherwise).  Enqueues a copy on
+ * the context's stream.
+ */
+asd_status asd_get_trajectory(asd_ctx* ctx, float* traj_dev);
+
+/*
+ * Run statistics of the Verifier (Algorithm 2): hist_host[m] = number of chain-rounds since the last
+ * asd_reset whose accepted prefix had length m (m = the chain's window means the whole window was
+ * accepted; a chain-round advances m + 1 steps otherwise), m = 0 .. min(capacity, window + 1) - 1;
+ * *n_out = entries written.  hist_host is a HOST buffer; the call synchronises the stream.
+ * Rounds of asd_sequential_ddpm count as prefix 1.
+ */
+asd_status asd_get_prefix_histogram(asd_ctx* ctx, int64_t* hist_host, int32_t capacity, int32_t* n_out);
 
 /*
  * The drift alone: out[r] = g(t_{step[r]}, y[r]) for r < n_rows, with the conditioning of

@@ -16,7 +16,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 EXPORTED_SYMBOLS = [
     "asd_version", "asd_create", "asd_reset", "asd_round", "asd_sample", "asd_sequential_ddpm",
     "asd_sample_host", "asd_get_state", "asd_set_state", "asd_get_window_state", "asd_set_window_state", "asd_debug_last_round", "asd_denoise",
-    "asd_set_profiling", "asd_get_profile", "asd_ddpm_schedule", "asd_debug_wait_selftest", "asd_denoise_static", "asd_denoise_static_max_rows",
+    "asd_set_profiling", "asd_get_profile", "asd_get_trajectory", "asd_get_prefix_histogram", "asd_ddpm_schedule", "asd_debug_wait_selftest", "asd_denoise_static", "asd_denoise_static_max_rows",
     "asd_last_error", "asd_destroy",
 ]
 
@@ -26,6 +26,8 @@ KIND = {"gmm": 0, "gauss": 1, "mlp": 2}
 FLAG_DEBUG_ALL_SLOTS = 1   # ASD_FLAG_DEBUG_ALL_SLOTS
 FLAG_ADAPTIVE_WINDOW = 2   # ASD_FLAG_ADAPTIVE_WINDOW
 FLAG_LOOKAHEAD = 4         # ASD_FLAG_LOOKAHEAD
+FLAG_TRAJECTORY = 8        # ASD_FLAG_TRAJECTORY
+FLAG_DEBUG_DUMP = 16       # ASD_FLAG_DEBUG_DUMP
 
 
 PRED = {"x0": 0, "eps": 1, "v": 2}
@@ -142,6 +144,8 @@ def load_library():
         "asd_get_window_state": [vp, vp, vp],
         "asd_set_window_state": [vp, vp, vp],
         "asd_debug_last_round": [vp, vp, vp, vp],
+        "asd_get_trajectory": [vp, vp],
+        "asd_get_prefix_histogram": [vp, vp, i32, C.POINTER(i32)],
         "asd_denoise": [vp, i32, vp, vp, vp, vp],
         "asd_denoise_static": [vp, i32, vp, vp, vp, vp],
         "asd_denoise_static_max_rows": [vp, C.POINTER(i32)],
@@ -338,6 +342,25 @@ class AsdSampler:
         acc = self._empty((self.n,), torch.int32)
         self._check(self.lib.asd_debug_last_round(self._ctx, _dev_ptr(lr), _dev_ptr(lu), _dev_ptr(acc)))
         return lr, lu, acc
+
+    def accepted_last_round(self):
+        """Accepted prefix length per chain in the last round (-1: the chain was not active)."""
+        acc = self._empty((self.n,), self._torch.int32)
+        self._check(self.lib.asd_debug_last_round(self._ctx, None, None, _dev_ptr(acc)))
+        return acc
+
+    def get_trajectory(self):
+        """(y_0 .. y_K) per chain, [n, K + 1, d]; needs FLAG_TRAJECTORY at construction."""
+        traj = self._empty((self.n, self.K + 1, self.d), self._torch.float32)
+        self._check(self.lib.asd_get_trajectory(self._ctx, _dev_ptr(traj)))
+        return traj
+
+    def prefix_histogram(self) -> np.ndarray:
+        """Chain-rounds since the last reset by accepted prefix length (index = length, 0 .. window)."""
+        h = np.zeros(min(self.window, self.K) + 1, dtype=np.int64)
+        n = C.c_int32(0)
+        self._check(self.lib.asd_get_prefix_histogram(self._ctx, _np_ptr(h), len(h), C.byref(n)))
+        return h[:n.value]
 
     def denoise(self, steps, y, slots=None):
         torch = self._torch

@@ -35,24 +35,32 @@ asd_status fail(Ctx* c, asd_status st, const std::string& msg) {
   } while (0)
 
 template <typename T>
-asd_status dev_alloc(Ctx* c, T** out, size_t count) {
+asd_status dev_alloc(Ctx* c, T** out, size_t count, bool zero = true) {
   void* p = nullptr;
   const size_t bytes = std::max<size_t>(count, 1) * sizeof(T);
   cudaError_t e = cudaMalloc(&p, bytes);
   if (e != cudaSuccess) return fail(c, ASD_ERR_OOM, std::string("cudaMalloc: ") + cudaGetErrorString(e));
   c->dev_allocs.push_back(p);
-  e = cudaMemsetAsync(p, 0, bytes, c->stream);
-  if (e != cudaSuccess) return fail(c, ASD_ERR_CUDA, std::string("cudaMemset: ") + cudaGetErrorString(e));
+  if (zero) {
+    e = cudaMemsetAsync(p, 0, bytes, c->stream);
+    if (e != cudaSuccess) return fail(c, ASD_ERR_CUDA, std::string("cudaMemset: ") + cudaGetErrorString(e));
+  }
   *out = static_cast<T*>(p);
   return ASD_OK;
 }
 
+// A table or parameter array that is written in full: no clearing, and the copy goes to the context's
+// stream like everything else the library enqueues (the stream may be a non-blocking one, which the
+// legacy default stream does not order against); the host vector may die right after the call.
 template <typename T>
 asd_status dev_upload(Ctx* c, const T** out, const std::vector<T>& host) {
   T* p = nullptr;
-  asd_status st = dev_alloc(c, &p, host.size());
+  asd_status st = dev_alloc(c, &p, host.size(), host.empty());
   if (st != ASD_OK) return st;
-  if (!host.empty()) ASD_CUDA(c, cudaMemcpy(p, host.data(), host.size() * sizeof(T), cudaMemcpyHostToDevice));
+  if (!host.empty()) {
+    ASD_CUDA(c, cudaMemcpyAsync(p, host.data(), host.size() * sizeof(T), cudaMemcpyHostToDevice, c->stream));
+    ASD_CUDA(c, cudaStreamSynchronize(c->stream));
+  }
   *out = p;
   return ASD_OK;
 }
@@ -276,8 +284,7 @@ asd_status enqueue_rounds(Ctx* c, bool graphs, int window, bool use_u, int activ
 // run is bound by the power cap, so what counts is energy per FLOP, not idle gaps.
 bool use_stagger(const Ctx* c) {
   if (c->kind != ASD_DEN_RESMLP_BF16 || !c->G2 || c->window < 4 || c->n < 2 || c->lookahead) return false;
-  const char* e = getenv("ASD_STAGGER");
-  return e && e[0] == '1';
+  return c->stagger;
 }
 
 // asd_sample for two staggered lanes: same run-ahead scheme as below, one ring slot per tick holding both
@@ -457,9 +464,11 @@ asd_status asd_create(const asd_config* cfg, void* cuda_stream, asd_ctx** out) {
   *out = nullptr;
   if (cfg->d < 1 || cfg->d > 65536) return bad(ASD_ERR_INVALID_ARG, "d must be in 1..65536");
   if (cfg->K < 1) return bad(ASD_ERR_INVALID_ARG, "K must be >= 1");
-  if (cfg->window < 1 || cfg->window > kMaxWindow) return bad(ASD_ERR_INVALID_ARG, "window must be in 1..64");
+  if (cfg->window < 1) return bad(ASD_ERR_INVALID_ARG, "window must be >= 1");
   if (cfg->max_chains < 1) return bad(ASD_ERR_INVALID_ARG, "max_chains must be >= 1");
-  if (cfg->flags & ~(ASD_FLAG_DEBUG_ALL_SLOTS | ASD_FLAG_ADAPTIVE_WINDOW | ASD_FLAG_LOOKAHEAD)) return bad(ASD_ERR_INVALID_ARG, "unknown flag");
+  if (cfg->flags & ~(ASD_FLAG_DEBUG_ALL_SLOTS | ASD_FLAG_ADAPTIVE_WINDOW | ASD_FLAG_LOOKAHEAD | ASD_FLAG_TRAJECTORY |
+                     ASD_FLAG_DEBUG_DUMP))
+    return bad(ASD_ERR_INVALID_ARG, "unknown flag");
   if (!cfg->t) return bad(ASD_ERR_INVALID_ARG, "t must not be NULL");
   if (!(cfg->t[0] >= 0.0)) return bad(ASD_ERR_INVALID_ARG, "t[0] must be >= 0");
   for (int i = 0; i < cfg->K; ++i) {
@@ -469,9 +478,12 @@ asd_status asd_create(const asd_config* cfg, void* cuda_stream, asd_ctx** out) {
       return bad(ASD_ERR_INVALID_ARG, "sigma2 must be finite and positive");
   }
   const bool lookahead = (cfg->flags & ASD_FLAG_LOOKAHEAD) != 0;
-  const long long max_rows_ll = (long long)cfg->max_chains * (lookahead ? cfg->window : std::max(cfg->window - 1, 1));
+  const int window_eff = std::min(cfg->window, cfg->K);  // a window beyond the grid acts like K (theta = infinity)
+  const long long max_rows_ll = (long long)cfg->max_chains * (lookahead ? window_eff : std::max(window_eff - 1, 1));
   if (max_rows_ll > (1ll << 30) || max_rows_ll * cfg->d > (1ll << 40))
     return bad(ASD_ERR_INVALID_ARG, "max_chains * window * d too large");
+  if ((cfg->flags & ASD_FLAG_TRAJECTORY) && (long long)cfg->max_chains * (cfg->K + 1ll) * cfg->d > (1ll << 36))
+    return bad(ASD_ERR_INVALID_ARG, "trajectory buffer (max_chains * (K + 1) * d floats) too large");
   const asd_denoiser& D = cfg->den;
   switch (D.kind) {
     case ASD_DEN_GMM_ISO:
@@ -531,6 +543,10 @@ asd_status asd_create(const asd_config* cfg, void* cuda_stream, asd_ctx** out) {
   {
     const char* e = getenv("ASD_GRAPHS");  // "0" launches every kernel of a round separately
     c->use_graphs = !(e && e[0] == '0');
+    const char* gm = getenv("ASD_GEMM_MODE");  // tuning aid: pins the GEMM kernel family
+    c->gemm_mode = !gm ? 0 : (!strcmp(gm, "cta") ? 1 : (!strcmp(gm, "pair") ? 2 : 0));
+    const char* sg = getenv("ASD_STAGGER");
+    c->stagger = sg && sg[0] == '1';
     if (cudaStreamCreateWithFlags(&c->gstream, cudaStreamNonBlocking) != cudaSuccess ||
         cudaEventCreateWithFlags(&c->fork_ev, cudaEventDisableTiming) != cudaSuccess ||
         cudaEventCreateWithFlags(&c->join_ev, cudaEventDisableTiming) != cudaSuccess)
@@ -588,9 +604,13 @@ asd_status asd_create(const asd_config* cfg, void* cuda_stream, asd_ctx** out) {
   TRY(dev_alloc(c, &c->v, n * d));
   TRY(dev_alloc(c, &c->Yhat, R * d));
   TRY(dev_alloc(c, &c->G, R * d));
-  TRY(dev_alloc(c, &c->dbg_lr, n * c->window));
-  TRY(dev_alloc(c, &c->dbg_lu, n * c->window));
+  if (cfg->flags & (ASD_FLAG_DEBUG_DUMP | ASD_FLAG_DEBUG_ALL_SLOTS)) {
+    TRY(dev_alloc(c, &c->dbg_lr, n * c->window));
+    TRY(dev_alloc(c, &c->dbg_lu, n * c->window));
+  }
   TRY(dev_alloc(c, &c->acc_len, n));
+  TRY(dev_alloc(c, &c->hist, (size_t)c->window + 1));
+  if (cfg->flags & ASD_FLAG_TRAJECTORY) TRY(dev_alloc(c, &c->traj, n * ((size_t)K + 1) * d));
   if (c->lookahead) {
     TRY(dev_alloc(c, &c->has_v, n));
     TRY(dev_alloc(c, &c->vsave, n * d));
@@ -676,9 +696,9 @@ asd_status asd_create(const asd_config* cfg, void* cuda_stream, asd_ctx** out) {
     TRY(dev_alloc(c, &M.X, (size_t)M.row_cap * M.in_pad));
     TRY(dev_alloc(c, &M.H[0], (size_t)M.row_cap * W));
     TRY(dev_alloc(c, &M.H[1], (size_t)M.row_cap * W));
-    TRY(dev_alloc(c, &c->G2, R * d));
+    if (c->stagger) TRY(dev_alloc(c, &c->G2, R * d));  // the staggered schedule alternates two drift buffers
     TRY(dev_alloc(c, &c->merged_rows, 4));
-    for (int l = 0; l < 2; ++l) {
+    for (int l = 0; l < 2 && c->stagger; ++l) {
       TRY(dev_alloc(c, &c->lanes[l].act, n));
       TRY(dev_alloc(c, &c->lanes[l].row_off, n + 1));
       TRY(dev_alloc(c, &c->lanes[l].step1, n));
@@ -718,6 +738,7 @@ asd_status asd_reset(asd_ctx* ctx, int32_t n_chains, uint64_t chain_id_base, con
   ASD_CUDA(c, cudaMemsetAsync(c->counters, 0, 2 * sizeof(RoundCounters), c->stream));
   launch_fill_int(c, c->acc_len, c->max_chains, -1);
   if (c->has_v) ASD_CUDA(c, cudaMemsetAsync(c->has_v, 0, (size_t)c->max_chains * sizeof(int), c->stream));
+  ASD_CUDA(c, cudaMemsetAsync(c->hist, 0, ((size_t)c->window + 1) * sizeof(unsigned long long), c->stream));
   if (c->G2) {
     const int h = (n_chains + 1) / 2;
     c->lanes[0].start = 0;
@@ -738,6 +759,7 @@ asd_status asd_reset(asd_ctx* ctx, int32_t n_chains, uint64_t chain_id_base, con
                                 cudaMemcpyDeviceToDevice, c->stream));
     launch_cond_to_bf16(c, n_chains);
   }
+  launch_traj_seed(c);  // y_0 is row 0 of every trajectory
   ASD_CUDA(c, cudaGetLastError());
   c->have_reset = true;
   c->round_bound = n_chains;
@@ -786,7 +808,8 @@ static asd_status finish_run(Ctx* c, float* y_out_dev, int32_t* rounds_out_dev, 
     stats->rounds_mean = 0.0;
     if (want_round_stats && c->n > 0) {
       std::vector<int> r(c->n);
-      ASD_CUDA(c, cudaMemcpy(r.data(), c->rounds, (size_t)c->n * sizeof(int), cudaMemcpyDeviceToHost));
+      ASD_CUDA(c, cudaMemcpyAsync(r.data(), c->rounds, (size_t)c->n * sizeof(int), cudaMemcpyDeviceToHost, c->stream));
+      ASD_CUDA(c, cudaStreamSynchronize(c->stream));
       long long sum = 0;
       int mx = 0;
       for (int v : r) {
@@ -992,6 +1015,7 @@ asd_status asd_set_state(asd_ctx* ctx, const int32_t* a_dev, const float* y_dev,
   if ((a_dev || y_dev) && c->has_v) ASD_CUDA(c, cudaMemsetAsync(c->has_v, 0, (size_t)c->max_chains * sizeof(int), c->stream));
   if (rounds_dev)
     ASD_CUDA(c, cudaMemcpyAsync(c->rounds, rounds_dev, (size_t)c->n * sizeof(int), cudaMemcpyDeviceToDevice, c->stream));
+  if (a_dev || y_dev) launch_traj_seed(c);  // the restored state is row a of the trajectory
   return ASD_OK;
 }
 
@@ -1018,10 +1042,36 @@ asd_status asd_debug_last_round(asd_ctx* ctx, float* ln_ratio_dev, float* ln_u_d
   Ctx* c = &ctx->c;
   if (!c->have_reset) return fail(c, ASD_ERR_STATE, "asd_debug_last_round before asd_reset");
   const size_t nw = (size_t)c->n * c->window;
+  if ((ln_ratio_dev || ln_u_dev) && !c->dbg_lr)
+    return fail(c, ASD_ERR_STATE, "ln ratio / ln u are recorded only by a context created with ASD_FLAG_DEBUG_DUMP");
   if (ln_ratio_dev) ASD_CUDA(c, cudaMemcpyAsync(ln_ratio_dev, c->dbg_lr, nw * sizeof(float), cudaMemcpyDeviceToDevice, c->stream));
   if (ln_u_dev) ASD_CUDA(c, cudaMemcpyAsync(ln_u_dev, c->dbg_lu, nw * sizeof(float), cudaMemcpyDeviceToDevice, c->stream));
   if (accepted_dev)
     ASD_CUDA(c, cudaMemcpyAsync(accepted_dev, c->acc_len, (size_t)c->n * sizeof(int), cudaMemcpyDeviceToDevice, c->stream));
+  return ASD_OK;
+}
+
+asd_status asd_get_trajectory(asd_ctx* ctx, float* traj_dev) {
+  if (!ctx) return ASD_ERR_INVALID_ARG;
+  Ctx* c = &ctx->c;
+  if (!c->have_reset) return fail(c, ASD_ERR_STATE, "asd_get_trajectory before asd_reset");
+  if (!c->traj) return fail(c, ASD_ERR_STATE, "the context was created without ASD_FLAG_TRAJECTORY");
+  if (!traj_dev) return fail(c, ASD_ERR_INVALID_ARG, "traj_dev must not be NULL");
+  ASD_CUDA(c, cudaMemcpyAsync(traj_dev, c->traj, (size_t)c->n * (c->K + 1) * c->d * sizeof(float), cudaMemcpyDeviceToDevice,
+                              c->stream));
+  return ASD_OK;
+}
+
+asd_status asd_get_prefix_histogram(asd_ctx* ctx, int64_t* hist_host, int32_t capacity, int32_t* n_out) {
+  if (!ctx) return ASD_ERR_INVALID_ARG;
+  Ctx* c = &ctx->c;
+  if (!hist_host || !n_out || capacity < 0) return fail(c, ASD_ERR_INVALID_ARG, "hist_host and n_out required");
+  if (!c->have_reset) return fail(c, ASD_ERR_STATE, "asd_get_prefix_histogram before asd_reset");
+  const int m = std::min(capacity, c->window + 1);
+  static_assert(sizeof(unsigned long long) == sizeof(int64_t), "histogram entries are 64 bit");
+  ASD_CUDA(c, cudaMemcpyAsync(hist_host, c->hist, (size_t)m * sizeof(int64_t), cudaMemcpyDeviceToHost, c->stream));
+  ASD_CUDA(c, cudaStreamSynchronize(c->stream));
+  *n_out = m;
   return ASD_OK;
 }
 

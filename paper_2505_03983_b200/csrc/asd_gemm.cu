@@ -1024,6 +1024,16 @@ bool get_tmap(Ctx* c, const void* ptr, int rows, int cols, int box_rows, CUtenso
   return true;
 }
 
+// The opt-in to more than 48 KB of dynamic shared memory is a per-device attribute of the kernel; a
+// context belongs to one device, so it remembers what it has set (the largest size asked for so far).
+void ensure_dynamic_smem(Ctx* c, const void* func, int bytes) {
+  int& have = c->func_smem[func];
+  if (bytes > have) {
+    cudaFuncSetAttribute(func, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    have = bytes;
+  }
+}
+
 template <int BN, int EPI>
 asd_status launch_gemm_t(Ctx* c, const void* a_ptr, int a_cols, const void* w_ptr, const GemmArgs& g, int m_bound) {
   using C = Cfg<BN>;
@@ -1032,11 +1042,7 @@ asd_status launch_gemm_t(Ctx* c, const void* a_ptr, int a_cols, const void* w_pt
     c->err = "cuTensorMapEncodeTiled failed";
     return ASD_ERR_CUDA;
   }
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaFuncSetAttribute(gemm_kernel<BN, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
-    attr_set = true;
-  }
+  ensure_dynamic_smem(c, reinterpret_cast<const void*>(&gemm_kernel<BN, EPI>), C::kSmemBytes);
   const int tiles = ((m_bound + BM - 1) / BM) * ((g.n_out + BN - 1) / BN);
   const int grid = tiles < c->num_sms ? (tiles < 1 ? 1 : tiles) : c->num_sms;
   gemm_kernel<BN, EPI><<<grid, kGemmThreads, C::kSmemBytes, c->stream>>>(ma, mw, g);
@@ -1052,11 +1058,7 @@ asd_status launch_gemm_pair_t(Ctx* c, const void* a_ptr, int a_cols, const void*
     c->err = "cuTensorMapEncodeTiled failed";
     return ASD_ERR_CUDA;
   }
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaFuncSetAttribute(gemm_pair_kernel<BN, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
-    attr_set = true;
-  }
+  ensure_dynamic_smem(c, reinterpret_cast<const void*>(&gemm_pair_kernel<BN, EPI>), C::kSmemBytes);
   const int tiles = ((m_bound + 2 * BM - 1) / (2 * BM)) * ((g.n_out + BN - 1) / BN);
   const int pairs = std::max(1, std::min(tiles, c->num_sms / 2));
   cudaLaunchConfig_t cfg = {};
@@ -1089,11 +1091,7 @@ asd_status launch_gemm_skinny(Ctx* c, const void* a_ptr, int a_cols, const void*
   const int budget = m_pad <= 128 ? kSkinnySmallBudget : kSkinnyStageBudget;
   const int stages = std::max(2, std::min(kSkinnyMaxStages, budget / skinny_stage_bytes(m_pad)));
   const int smem = std::max(stages * skinny_stage_bytes(m_pad), m_pad * BM * 4) + 1024 + 256;
-  static int attr_smem = 0;
-  if (smem > attr_smem) {
-    cudaFuncSetAttribute(gemm_skinny_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-    attr_smem = smem;
-  }
+  ensure_dynamic_smem(c, reinterpret_cast<const void*>(&gemm_skinny_kernel<EPI>), smem);
   const dim3 grid(((g.n_out + BM - 1) / BM) * kSplit, row_blocks);
   // Programmatic dependent launch: this kernel may begin (barriers, tensor memory, first weight tiles)
   // while the previous kernel of the stream is still finishing; it waits for it before it touches
@@ -1116,12 +1114,9 @@ asd_status launch_gemm_skinny(Ctx* c, const void* a_ptr, int a_cols, const void*
   return ASD_OK;
 }
 
-// Few rows: weight streaming with swapped operands.  (ASD_GEMM_MODE=cta|pair pins the tiled kernels.)
-bool use_skinny(int m_bound) {
-  const char* e = getenv("ASD_GEMM_MODE");
-  const bool pinned = e && (!strcmp(e, "cta") || !strcmp(e, "pair"));
-  return !pinned && m_bound <= kSkinnyMaxRows;
-}
+// Few rows: weight streaming with swapped operands.  (ASD_GEMM_MODE=cta|pair, read at asd_create, pins the
+// tiled kernels.)
+bool use_skinny(const Ctx* c, int m_bound) { return c->gemm_mode == 0 && m_bound <= kSkinnyMaxRows; }
 
 // Which kernel and column-tile width serve a [m x k] x [n x k]^T product best.  Model: every SM fills
 // its shared memory from L2 at about 50 bytes per clock and its tensor pipe retires a 128 x 256 x 64
@@ -1132,8 +1127,7 @@ struct GemmPlan {
 };
 
 GemmPlan plan_gemm(const Ctx* c, int m_bound, int n_out) {
-  const char* e = getenv("ASD_GEMM_MODE");  // tuning aid: "cta" or "pair" pins the kernel family
-  const int mode = !e ? 0 : (!strcmp(e, "cta") ? 1 : (!strcmp(e, "pair") ? 2 : 0));
+  const int mode = c->gemm_mode;  // tuning aid: 1 ("cta") or 2 ("pair") pins the kernel family
   const double fill_rate = 50.0;
   GemmPlan best{false, 32};
   double best_t = 1e300;
@@ -1161,7 +1155,7 @@ GemmPlan plan_gemm(const Ctx* c, int m_bound, int n_out) {
 
 template <int EPI>
 asd_status launch_gemm(Ctx* c, const void* a_ptr, int a_cols, const void* w_ptr, const GemmArgs& g, int m_bound) {
-  if (use_skinny(m_bound)) return launch_gemm_skinny<EPI>(c, a_ptr, a_cols, w_ptr, g, m_bound);
+  if (use_skinny(c, m_bound)) return launch_gemm_skinny<EPI>(c, a_ptr, a_cols, w_ptr, g, m_bound);
   const GemmPlan p = plan_gemm(c, m_bound, g.n_out);
   if (p.pair) {
     switch (p.bn) {
@@ -1208,18 +1202,18 @@ asd_status mlp_forward(Ctx* c, const RowSet& rs, float* out, int pass) {
     st = launch_gemm<EPI_IN>(c, M.X, M.in_pad, M.W_in, g, m_bound);
   }
   if (st != ASD_OK) return st;
-  ProfScope ps_hid(pass < 2 ? c : nullptr, ph_hid);
-  // residual layers
-  for (int l = 0; l < M.n_layers; ++l) {
-    g.k_dim = M.width;
-    g.bias = M.b_hid + (size_t)l * M.width;
-    g.resid = M.H[l & 1];
-    g.out_bf16 = M.H[(l + 1) & 1];
-    st = launch_gemm<EPI_HID>(c, M.H[l & 1], M.width, M.W_hid + (size_t)l * M.width * M.width, g, m_bound);
-    if (st != ASD_OK) return st;
+  {
+    ProfScope ps(pass < 2 ? c : nullptr, ph_hid);
+    // residual layers
+    for (int l = 0; l < M.n_layers; ++l) {
+      g.k_dim = M.width;
+      g.bias = M.b_hid + (size_t)l * M.width;
+      g.resid = M.H[l & 1];
+      g.out_bf16 = M.H[(l + 1) & 1];
+      st = launch_gemm<EPI_HID>(c, M.H[l & 1], M.width, M.W_hid + (size_t)l * M.width * M.width, g, m_bound);
+      if (st != ASD_OK) return st;
+    }
   }
-  ps_hid.~ProfScope();
-  ps_hid.c = nullptr;
   // output projection with the skip / scale epilogue
   g.n_out = c->d;
   g.k_dim = M.width;

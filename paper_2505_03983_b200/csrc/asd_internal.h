@@ -16,7 +16,6 @@
 
 namespace asd {
 
-constexpr int kMaxWindow = 64;  // speculation length limit (two ballots in the verify kernel)
 
 // ---- device-side bookkeeping shared by all kernels of a round -------------------------
 // One small block of counters in device memory; the prep kernel rewrites it every round.
@@ -158,9 +157,11 @@ struct Ctx {
   Lane lanes[2];
   int* merged_rows = nullptr;
   long long extra_rows_total = 0, extra_rows_verified = 0;  // lanes' counters, added by the run statistics
-  float* dbg_lr = nullptr;   // [max_chains, window]
+  float* dbg_lr = nullptr;   // [max_chains, window]  (ASD_FLAG_DEBUG_DUMP / ASD_FLAG_DEBUG_ALL_SLOTS only)
   float* dbg_lu = nullptr;   // [max_chains, window]
   int* acc_len = nullptr;    // [max_chains]
+  float* traj = nullptr;     // [max_chains, K + 1, d] (ASD_FLAG_TRAJECTORY only)
+  unsigned long long* hist = nullptr;  // [window + 1] chain-rounds by accepted prefix length since the last reset
   RoundCounters* counters = nullptr;
   RoundCounters* counters_host = nullptr;  // pinned
   // asd_sample runs ahead of the device: the counters of round r land in ring_host[r % kRing] and
@@ -175,6 +176,9 @@ struct Ctx {
   MlpParams mlp{};
   std::vector<void*> dev_allocs;
   std::map<std::tuple<const void*, int, int, int>, CUtensorMap> tmaps;
+  std::map<const void*, int> func_smem;  // kernel -> dynamic shared memory opted in on this context's device
+  int gemm_mode = 0;                     // ASD_GEMM_MODE at asd_create: 0 planner, 1 "cta", 2 "pair"
+  bool stagger = false;                  // ASD_STAGGER=1 at asd_create
   // One speculation round captured as a CUDA graph per (window, use_u, bound on active chains); replayed
   // on a private stream that is forked from and joined to the caller's stream.
   struct RoundGraph { cudaGraphExec_t exec; long long launches; };
@@ -221,6 +225,7 @@ void launch_gmm(Ctx* c, const RowSet& rs, float* out);
 void launch_gauss(Ctx* c, const RowSet& rs, float* out);
 void launch_cond_to_bf16(Ctx* c, int n);
 void launch_fill_int(Ctx* c, int* p, int n, int val);
+void launch_traj_seed(Ctx* c);  // trajectory row a_j <- y_j for every chain of the batch
 
 // ---- MLP forward (asd_gemm.cu) ----------------------------------------------------------
 // Runs the GEMM chain on the rows already packed into mlp.X; writes out[r] for r < *n_rows_dev.

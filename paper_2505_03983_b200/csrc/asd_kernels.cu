@@ -280,6 +280,7 @@ struct DraftArgs {
 
 constexpr int kDraftQ = 32;       // float4 groups (= 128 dims) per block
 constexpr int kDraftThreads = 256;
+constexpr int kDraftChunk = 64;   // slots staged in shared memory at a time (staged form); longer windows take several chunks
 
 // fp32 point and (network denoiser) bf16 input of row `row`, slot k, for float4 group q
 __device__ __forceinline__ void draft_store(const DraftArgs& A, int row, int a, int k, int q, float4 yh) {
@@ -305,7 +306,7 @@ __device__ __forceinline__ void draft_store(const DraftArgs& A, int row, int a, 
 }
 
 __global__ void __launch_bounds__(kDraftThreads) draft_kernel(const DraftArgs A) {
-  __shared__ float4 s_pt[kMaxWindow][kDraftQ];  // noise, then drafted points, per slot (parallel form)
+  __shared__ float4 s_pt[kDraftChunk][kDraftQ];  // noise, then drafted points, per slot of a chunk (parallel form)
   const int p = blockIdx.x;
   if (p >= A.cnt->n_active) return;
   const int j = A.act[p];
@@ -334,31 +335,39 @@ __global__ void __launch_bounds__(kDraftThreads) draft_kernel(const DraftArgs A)
       }
     }
   } else {
-    // small batches: the noise of all slots in parallel, then the recurrence by one warp, then the stores
+    // small batches: the noise of a chunk of slots in parallel, then the recurrence by one warp (which carries
+    // the point from chunk to chunk in registers), then the stores
     const int ql = threadIdx.x & (kDraftQ - 1), ks = threadIdx.x / kDraftQ;
     constexpr int kSlotLanes = kDraftThreads / kDraftQ;
     const int q = blockIdx.y * kDraftQ + ql;
     const bool q_ok = q < A.nq;
-    if (q_ok)
-      for (int k = 1 + ks; k <= nr; k += kSlotLanes) s_pt[k - 1][ql] = xi4((uint32_t)q, (uint32_t)(a + k), chain, A.keys);
-    __syncthreads();
+    float4 yh = make_float4(0.f, 0.f, 0.f, 0.f), v = yh;
     if (ks == 0 && q_ok) {
-      float4 yh = load4(A.y + (size_t)j * A.d, q, A.d, A.vec);
-      const float4 v = load4(vrow, q, A.d, A.vec);
-      for (int k = 1; k <= nr; ++k) {
-        const int i = a + k - 1;
-        const float eta = A.tab.eta[i], sig = A.tab.sig[i];
-        const float4 xi = s_pt[k - 1][ql];
-        yh.x = fmaf(sig, xi.x, fmaf(eta, v.x, yh.x));
-        yh.y = fmaf(sig, xi.y, fmaf(eta, v.y, yh.y));
-        yh.z = fmaf(sig, xi.z, fmaf(eta, v.z, yh.z));
-        yh.w = fmaf(sig, xi.w, fmaf(eta, v.w, yh.w));
-        s_pt[k - 1][ql] = yh;
-      }
+      yh = load4(A.y + (size_t)j * A.d, q, A.d, A.vec);
+      v = load4(vrow, q, A.d, A.vec);
     }
-    __syncthreads();
-    if (q_ok)
-      for (int k = 1 + ks; k <= nr; k += kSlotLanes) draft_store(A, row0 + k - 1, a, k, q, s_pt[k - 1][ql]);
+    for (int kc = 0; kc < nr; kc += kDraftChunk) {
+      const int kn = min(kDraftChunk, nr - kc);  // slots kc + 1 .. kc + kn
+      if (q_ok)
+        for (int kk = ks; kk < kn; kk += kSlotLanes) s_pt[kk][ql] = xi4((uint32_t)q, (uint32_t)(a + kc + kk + 1), chain, A.keys);
+      __syncthreads();
+      if (ks == 0 && q_ok) {
+        for (int kk = 0; kk < kn; ++kk) {
+          const int i = a + kc + kk;
+          const float eta = A.tab.eta[i], sig = A.tab.sig[i];
+          const float4 xi = s_pt[kk][ql];
+          yh.x = fmaf(sig, xi.x, fmaf(eta, v.x, yh.x));
+          yh.y = fmaf(sig, xi.y, fmaf(eta, v.y, yh.y));
+          yh.z = fmaf(sig, xi.z, fmaf(eta, v.z, yh.z));
+          yh.w = fmaf(sig, xi.w, fmaf(eta, v.w, yh.w));
+          s_pt[kk][ql] = yh;
+        }
+      }
+      __syncthreads();
+      if (q_ok)
+        for (int kk = ks; kk < kn; kk += kSlotLanes) draft_store(A, row0 + kc + kk, a, kc + kk + 1, q, s_pt[kk][ql]);
+      __syncthreads();
+    }
   }
   // row maps, conditioning, time embedding and zero padding: the chain's blocks share the slots (this block takes
   // slots k = 1 + blockIdx.y + i * gridDim.y).  With few blocks in flight (the staged form) the (slot, element) pairs
@@ -495,16 +504,24 @@ struct VerifyArgs {
   const float* Yhat;
   const float* G;
   Tables tab;
-  float* dbg_lr;
+  float* dbg_lr;   // diagnostics (ASD_FLAG_DEBUG_DUMP), else null
   float* dbg_lu;
   int* acc_len;
+  float* traj;     // [n, K + 1, d] states y_0 .. y_K (ASD_FLAG_TRAJECTORY), else null
+  unsigned long long* hist;  // [window + 1] chain-rounds by accepted prefix length
 };
 
 constexpr int kVerifyMaxWarps = 8;
 
+// ln ratio of Algorithm 3 from the two reductions, with the rounding of every operation spelled out so
+// that every kernel that evaluates it gets the same bits: -(eta/sigma) <xi, delta> - (eta^2 / 2 sigma^2) |delta|^2.
+__device__ __forceinline__ float ln_ratio_of(float c1, float c2, float dot, float nrm) {
+  return __fmaf_rn(-c1, dot, -__fmul_rn(c2, nrm));
+}
+
 __global__ void __launch_bounds__(256) verify_kernel(const VerifyArgs A) {
   __shared__ float s_part[2][kVerifyMaxWarps][2][kVerifyMaxWarps];  // [group parity][slot][dot | nrm][warp of team]
-  __shared__ float s_lu[kMaxWindow + 1];
+  __shared__ float s_lu[2][kVerifyMaxWarps];                        // [group parity][slot] ln u
   const int p = blockIdx.x;
   if (p >= A.cnt->n_active) return;
   const int j = A.act[p];
@@ -515,17 +532,16 @@ __global__ void __launch_bounds__(256) verify_kernel(const VerifyArgs A) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
   const float* vrow = (A.la && A.idx1[p] < 0) ? A.vsave + (size_t)j * A.d
                                                : A.v + (size_t)((A.la ? A.idx1[p] : (A.v_off ? *A.v_off : 0) + p)) * A.d;
-  const float nan = __int_as_float(0x7fc00000);
 
-  // ln u of every slot (one Philox call each), and the diagnostics of slot 1: proposal mean == target
-  // mean, ratio exactly 1 (Lemma 1)
-  for (int k = 1 + tid; k <= w; k += blockDim.x) {
-    const float lu = A.use_u ? ln_u((uint32_t)(a + k), chain, A.keys) : 0.f;
-    s_lu[k] = lu;
-    A.dbg_lu[(size_t)j * A.dbg_stride + k - 1] = lu;
-    A.dbg_lr[(size_t)j * A.dbg_stride + k - 1] = k == 1 ? 0.f : nan;
+  // diagnostics: ln u of every slot, and ln ratio = 0 for slot 1 (proposal mean == target mean, Lemma 1),
+  // NaN for the slots the walk below does not reach
+  if (A.dbg_lr) {
+    const float nan = __int_as_float(0x7fc00000);
+    for (int k = 1 + tid; k <= w; k += blockDim.x) {
+      A.dbg_lu[(size_t)j * A.dbg_stride + k - 1] = A.use_u ? ln_u((uint32_t)(a + k), chain, A.keys) : 0.f;
+      A.dbg_lr[(size_t)j * A.dbg_stride + k - 1] = k == 1 ? 0.f : nan;
+    }
   }
-  __syncthreads();
 
   // Slots are taken in groups of S = nwarps / wps; a team of wps warps reduces one slot.
   const int wps = A.wps, S = nwarps / wps;
@@ -537,6 +553,8 @@ __global__ void __launch_bounds__(256) verify_kernel(const VerifyArgs A) {
   for (int k0 = 2; k0 <= w; k0 += S, par ^= 1) {
     const int k = k0 + sw;
     rows_read = min(k0 + S - 1, w) - 1;
+    // ln u of the group's slots (one Philox call each), by the first S threads
+    if (tid < S && k0 + tid <= w) s_lu[par][tid] = A.use_u ? ln_u((uint32_t)(a + k0 + tid), chain, A.keys) : 0.f;
     float dot = 0.f, nrm = 0.f;
     if (k <= w) {
       const float* grow = A.G + (size_t)(row0 + k - 2) * A.d;
@@ -591,9 +609,9 @@ __global__ void __launch_bounds__(256) verify_kernel(const VerifyArgs A) {
         n2 += s_part[par][s2][1][x];
       }
       const int kk = k0 + s2, i = a + kk - 1;
-      const float lr = -A.tab.c1[i] * d2 - A.tab.c2[i] * n2;
-      const bool acc = (s_lu[kk] <= fminf(0.f, lr)) || (n2 == 0.f);
-      if (tid == 0) A.dbg_lr[(size_t)j * A.dbg_stride + kk - 1] = lr;
+      const float lr = ln_ratio_of(A.tab.c1[i], A.tab.c2[i], d2, n2);
+      const bool acc = (s_lu[par][s2] <= fminf(0.f, lr)) || (n2 == 0.f);
+      if (tid == 0 && A.dbg_lr) A.dbg_lr[(size_t)j * A.dbg_stride + kk - 1] = lr;
       if (!acc && n == w) {
         n = kk - 1;
         rej_dot = d2;
@@ -656,11 +674,24 @@ __global__ void __launch_bounds__(256) verify_kernel(const VerifyArgs A) {
     }
     if (tid == 0) A.has_v[j] = reuse ? 1 : 0;
   }
+  if (A.traj) {
+    // Algorithm 1's return value: the accepted proposal samples y^_{a+1} .. and, last, the new state
+    // (the reflected sample, or the end of a fully accepted window) become y_{a+1} .. y_{a+adv}
+    const int adv = (n < w) ? n + 1 : w;
+    float* tbase = A.traj + ((size_t)j * (A.K + 1) + a) * A.d;
+    __syncthreads();  // this block's stores to yrow are visible to all its threads
+    for (int k = 1; k <= adv; ++k) {
+      const float* src = (k < adv) ? A.Yhat + (size_t)(row0 + k - 1) * A.d : yrow;
+      float* dst = tbase + (size_t)k * A.d;
+      for (int e = tid; e < A.d; e += blockDim.x) dst[e] = src[e];
+    }
+  }
   if (tid == 0) {
     const int adv = (n < w) ? n + 1 : w;
     A.a[j] = a + adv;
     A.rounds[j] += 1;
     A.acc_len[j] = n;
+    if (A.hist) atomicAdd(&A.hist[n], 1ull);
     if (A.wnd) {
       // next speculation length of this chain: 2 + 1.5 x running mean of the steps it advances per round
       const int e8 = (A.ema8[j] + 8 * adv) >> 1;
@@ -705,9 +736,11 @@ void launch_verify(Ctx* c, const Lane& L, int window, bool use_u, const float* G
   A.Yhat = c->Yhat;
   A.G = G;
   A.tab = c->tab;
-  A.dbg_lr = c->dbg_lr + (size_t)L.start * c->window;
-  A.dbg_lu = c->dbg_lu + (size_t)L.start * c->window;
+  A.dbg_lr = c->dbg_lr ? c->dbg_lr + (size_t)L.start * c->window : nullptr;
+  A.dbg_lu = c->dbg_lu ? c->dbg_lu + (size_t)L.start * c->window : nullptr;
   A.acc_len = c->acc_len + L.start;
+  A.traj = c->traj ? c->traj + (size_t)L.start * (c->K + 1) * c->d : nullptr;
+  A.hist = c->hist;
   // eight warps per chain; a slot is reduced by two warps when a row has >= 512 float4 groups, else by one
   A.wps = A.nq >= 512 ? 2 : 1;
   verify_kernel<<<L.n, 256, 0, c->stream>>>(A);
@@ -886,6 +919,22 @@ void launch_cond_to_bf16(Ctx* c, int n) {
   int blocks = (int)((total + 255) / 256);
   blocks = blocks > 1024 ? 1024 : blocks;
   cond_to_bf16_kernel<<<blocks, 256, 0, c->stream>>>(c->cond_f32, const_cast<__nv_bfloat16*>(c->mlp.cond), total);
+  c->launches++;
+}
+
+// Trajectory bookkeeping: the state a chain is (re)started from is row a of its trajectory.
+__global__ void traj_seed_kernel(const int* __restrict__ a, const float* __restrict__ y, float* __restrict__ traj, int n,
+                                 int K, int d) {
+  for (int j = blockIdx.x; j < n; j += gridDim.x) {
+    const int aj = min(max(a[j], 0), K);
+    float* dst = traj + ((size_t)j * (K + 1) + aj) * d;
+    for (int e = threadIdx.x; e < d; e += blockDim.x) dst[e] = y[(size_t)j * d + e];
+  }
+}
+
+void launch_traj_seed(Ctx* c) {
+  if (!c->traj || c->n <= 0) return;
+  traj_seed_kernel<<<std::min(c->n, 8 * c->num_sms), 256, 0, c->stream>>>(c->a, c->y, c->traj, c->n, c->K, c->d);
   c->launches++;
 }
 

@@ -145,3 +145,26 @@ def test_resmlp_matches_plain_loops():
         # identical rounding points; a bf16 flip from summation order would show as ~4e-3 relative
         assert np.allclose(got, out, rtol=1e-9, atol=1e-9), np.abs(got - np.array(out)).max()
         assert np.allclose(g.batch([i], y[None], chain)[0], got, rtol=1e-9, atol=1e-9)
+
+
+@pytest.mark.parametrize("name", ["mlp_tiny", "mlp_ragged"])
+def test_resmlp_batch_rows_match_single_calls_mixed_steps(name):
+    """`batch` (one matrix product per layer over several points) against `__call__` row by row, with a
+    different step in every row: a row must get its own step's c_in, time embedding, c_skip and c_out, and
+    the conditioning of the chain it is called for."""
+    wl = workloads.make(name)
+    g = den.from_workload(wl)
+    rng = np.random.default_rng(8)
+    for chain in (0, wl.chains - 1):
+        steps = [0, wl.K - 1, 3, 3, wl.K // 2, 1, wl.K - 2]
+        Y = np.stack([rng.standard_normal(wl.d) * (1 + wl.t[i]) for i in steps])
+        got = g.batch(steps, Y, chain)
+        assert got.shape == (len(steps), wl.d)
+        for r, i in enumerate(steps):
+            one = g(i, Y[r], chain)
+            # same rounding points row by row; only the summation order inside the products may differ
+            assert np.allclose(got[r], one, rtol=1e-9, atol=1e-9), (r, np.abs(got[r] - one).max())
+        # the rows really are different functions of the step and the chain
+        assert not np.allclose(g.batch([5] * len(steps), Y, chain), got)
+        if wl.d_cond:
+            assert not np.allclose(g.batch(steps, Y, (chain + 1) % wl.chains), got)

@@ -143,8 +143,9 @@ def _mlp(name, d, d_cond, d_temb, width, n_layers, K, window, chains, seed,
 
 
 def make(name: str, *, chains: Optional[int] = None, K: Optional[int] = None,
-         window: Optional[int] = None, seed: Optional[int] = None) -> Workload:
-    """Build a named workload; keyword arguments override chains / K / window / seed."""
+         window: Optional[int] = None, seed: Optional[int] = None, n_layers: Optional[int] = None) -> Workload:
+    """Build a named workload; keyword arguments override chains / K / window / seed and, for the
+    network workloads, the number of residual layers (the other shapes stay)."""
     def ov(val, default):
         return default if val is None else val
 
@@ -154,12 +155,12 @@ def make(name: str, *, chains: Optional[int] = None, K: Optional[int] = None,
     if name == "cfg2_gauss64":
         return _gauss(name, 64, ov(K, 1000), ov(window, 16), ov(chains, 256), s)
     if name == "cfg3_policy":
-        return _mlp(name, 112, 64, 128, 1024, 4, ov(K, 100), ov(window, 16), ov(chains, 64), s)
+        return _mlp(name, 112, 64, 128, 1024, ov(n_layers, 4), ov(K, 100), ov(window, 16), ov(chains, 64), s)
     if name == "cfg4_image":
-        return _mlp(name, 3072, 0, 256, 4096, 6, ov(K, 1000), ov(window, 32), ov(chains, 32), s)
+        return _mlp(name, 3072, 0, 256, 4096, ov(n_layers, 6), ov(K, 1000), ov(window, 32), ov(chains, 32), s)
     m = re.fullmatch(r"sweep_b(\d+)_w(\d+)", name)
     if m:
-        return _mlp(name, 3072, 0, 256, 4096, 6, ov(K, 1000), ov(window, int(m.group(2))),
+        return _mlp(name, 3072, 0, 256, 4096, ov(n_layers, 6), ov(K, 1000), ov(window, int(m.group(2))),
                     ov(chains, int(m.group(1))), s)
     if name == "mlp_tiny":
         return _mlp(name, 24, 8, 32, 128, 2, ov(K, 40), ov(window, 6), ov(chains, 5), s, bias_std=0.05)
