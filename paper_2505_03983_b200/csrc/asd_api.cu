@@ -19,7 +19,6 @@ struct asd_ctx {
 namespace {
 
 thread_local std::string g_create_error;
-constexpr int kAdaptInitEma8 = 32;
 
 asd_status fail(Ctx* c, asd_status st, const std::string& msg) {
   if (c) c->err = msg;
@@ -547,6 +546,8 @@ asd_status asd_create(const asd_config* cfg, void* cuda_stream, asd_ctx** out) {
     c->gemm_mode = !gm ? 0 : (!strcmp(gm, "cta") ? 1 : (!strcmp(gm, "pair") ? 2 : 0));
     const char* sg = getenv("ASD_STAGGER");
     c->stagger = sg && sg[0] == '1';
+    const char* rm = getenv("ASD_RESIDENT");  // tuning aid: "0" keeps the closed-form drifts on the per-phase kernels
+    c->resident_mode = !rm ? 1 : (rm[0] == '0' ? 0 : (rm[0] == '2' ? 2 : 1));
     if (cudaStreamCreateWithFlags(&c->gstream, cudaStreamNonBlocking) != cudaSuccess ||
         cudaEventCreateWithFlags(&c->fork_ev, cudaEventDisableTiming) != cudaSuccess ||
         cudaEventCreateWithFlags(&c->join_ev, cudaEventDisableTiming) != cudaSuccess)
@@ -692,7 +693,6 @@ asd_status asd_create(const asd_config* cfg, void* cuda_stream, asd_ctx** out) {
     __nv_bfloat16* p = nullptr;
     TRY(dev_alloc(c, &p, n * (size_t)D.d_cond));
     M.cond = p;
-    TRY(dev_alloc(c, &c->cond_f32, n * (size_t)D.d_cond));
     TRY(dev_alloc(c, &M.X, (size_t)M.row_cap * M.in_pad));
     TRY(dev_alloc(c, &M.H[0], (size_t)M.row_cap * W));
     TRY(dev_alloc(c, &M.H[1], (size_t)M.row_cap * W));
@@ -728,17 +728,8 @@ asd_status asd_reset(asd_ctx* ctx, int32_t n_chains, uint64_t chain_id_base, con
   }
   c->n = n_chains;
   c->chain_base = chain_id_base;
-  const size_t nd = (size_t)n_chains * c->d;
-  if (y0_dev)
-    ASD_CUDA(c, cudaMemcpyAsync(c->y, y0_dev, nd * sizeof(float), cudaMemcpyDeviceToDevice, c->stream));
-  else
-    ASD_CUDA(c, cudaMemsetAsync(c->y, 0, nd * sizeof(float), c->stream));
-  ASD_CUDA(c, cudaMemsetAsync(c->a, 0, (size_t)c->max_chains * sizeof(int), c->stream));
-  ASD_CUDA(c, cudaMemsetAsync(c->rounds, 0, (size_t)c->max_chains * sizeof(int), c->stream));
-  ASD_CUDA(c, cudaMemsetAsync(c->counters, 0, 2 * sizeof(RoundCounters), c->stream));
-  launch_fill_int(c, c->acc_len, c->max_chains, -1);
-  if (c->has_v) ASD_CUDA(c, cudaMemsetAsync(c->has_v, 0, (size_t)c->max_chains * sizeof(int), c->stream));
-  ASD_CUDA(c, cudaMemsetAsync(c->hist, 0, ((size_t)c->window + 1) * sizeof(unsigned long long), c->stream));
+  // state, cursors, round and per-call counters, window state, histogram, trajectory row 0, bf16 conditioning
+  launch_reset(c, y0_dev, need_cond && n_chains > 0 ? cond_dev : nullptr);
   if (c->G2) {
     const int h = (n_chains + 1) / 2;
     c->lanes[0].start = 0;
@@ -751,15 +742,6 @@ asd_status asd_reset(asd_ctx* ctx, int32_t n_chains, uint64_t chain_id_base, con
     }
     ASD_CUDA(c, cudaMemsetAsync(c->merged_rows, 0, sizeof(int), c->stream));
   }
-  // adaptive mode starts every chain at 8 x mean = 32, i.e. a speculation length of min(window, 8)
-  launch_fill_int(c, c->ema8, c->max_chains, kAdaptInitEma8);
-  launch_fill_int(c, c->wnd, c->max_chains, std::max(2, std::min(c->window, 2 + (3 * kAdaptInitEma8) / 16)));
-  if (need_cond && n_chains > 0) {
-    ASD_CUDA(c, cudaMemcpyAsync(c->cond_f32, cond_dev, (size_t)n_chains * c->mlp.d_cond * sizeof(float),
-                                cudaMemcpyDeviceToDevice, c->stream));
-    launch_cond_to_bf16(c, n_chains);
-  }
-  launch_traj_seed(c);  // y_0 is row 0 of every trajectory
   ASD_CUDA(c, cudaGetLastError());
   c->have_reset = true;
   c->round_bound = n_chains;
@@ -772,7 +754,11 @@ asd_status asd_round(asd_ctx* ctx, asd_round_stats* stats_host) {
   Ctx* c = &ctx->c;
   if (!c->have_reset) return fail(c, ASD_ERR_STATE, "asd_round before asd_reset");
   // the bound on the active chains that sizes the grids: what the previous round reported, if it was read
-  asd_status st = enqueue_round(c, c->window, true, std::min(c->n, c->round_bound));
+  asd_status st;
+  if (c->resident_mode == 2 && !c->prof_on && resident_supported(c, c->window, nullptr))
+    st = launch_resident(c, c->window, true, 1);  // one round of the chain-resident kernel (lock-step tests)
+  else
+    st = enqueue_round(c, c->window, true, std::min(c->n, c->round_bound));
   if (st != ASD_OK) return st;
   if (stats_host) {
     st = sync_counters(c);
@@ -790,10 +776,8 @@ asd_status asd_round(asd_ctx* ctx, asd_round_stats* stats_host) {
 
 static asd_status finish_run(Ctx* c, float* y_out_dev, int32_t* rounds_out_dev, asd_run_stats* stats, long long launches0,
                              bool want_round_stats) {
-  if (y_out_dev)
-    ASD_CUDA(c, cudaMemcpyAsync(y_out_dev, c->y, (size_t)c->n * c->d * sizeof(float), cudaMemcpyDeviceToDevice, c->stream));
-  if (rounds_out_dev)
-    ASD_CUDA(c, cudaMemcpyAsync(rounds_out_dev, c->rounds, (size_t)c->n * sizeof(int), cudaMemcpyDeviceToDevice, c->stream));
+  launch_finish(c, y_out_dev, rounds_out_dev);  // results out, max / mean of the round counters into the counters
+  ASD_CUDA(c, cudaGetLastError());
   ASD_CUDA(c, cudaEventRecord(c->ev1, c->stream));
   asd_status st = sync_counters(c);
   if (st != ASD_OK) return st;
@@ -807,17 +791,8 @@ static asd_status finish_run(Ctx* c, float* y_out_dev, int32_t* rounds_out_dev, 
     stats->rounds_max = 0;
     stats->rounds_mean = 0.0;
     if (want_round_stats && c->n > 0) {
-      std::vector<int> r(c->n);
-      ASD_CUDA(c, cudaMemcpyAsync(r.data(), c->rounds, (size_t)c->n * sizeof(int), cudaMemcpyDeviceToHost, c->stream));
-      ASD_CUDA(c, cudaStreamSynchronize(c->stream));
-      long long sum = 0;
-      int mx = 0;
-      for (int v : r) {
-        sum += v;
-        mx = std::max(mx, v);
-      }
-      stats->rounds_max = mx;
-      stats->rounds_mean = (double)sum / c->n;
+      stats->rounds_max = c->counters_host->rounds_max;
+      stats->rounds_mean = (double)c->counters_host->rounds_sum / c->n;
     }
   }
   return ASD_OK;
@@ -835,6 +810,13 @@ asd_status asd_sample(asd_ctx* ctx, float* y_out_dev, int32_t* rounds_out_dev, a
   // upper bound (chains only finish), and the rounds enqueued after the last chain finished find no
   // active chain and do nothing.  Theorem 3: the cursor strictly increases, so K rounds always suffice.
   c->extra_rows_total = c->extra_rows_verified = 0;
+  // Closed-form drifts: the whole while loop of every chain inside one launch, a block per chain.
+  if (c->resident_mode >= 1 && !c->prof_on && resident_supported(c, c->window, nullptr)) {
+    asd_status st = launch_resident(c, c->window, true, 0x7fffffff);
+    if (st != ASD_OK) return st;
+    ASD_CUDA(c, cudaGetLastError());
+    return finish_run(c, y_out_dev, rounds_out_dev, stats_host, launches0, true);
+  }
   if (use_stagger(c)) {
     asd_status st = sample_staggered(c);
     if (st != ASD_OK) return st;
@@ -909,6 +891,13 @@ asd_status asd_sequential_ddpm(asd_ctx* ctx, float* y_out_dev, asd_run_stats* st
   Ctx* c = &ctx->c;
   if (!c->have_reset) return fail(c, ASD_ERR_STATE, "asd_sequential_ddpm before asd_reset");
   const long long launches0 = c->launches;
+  if (c->resident_mode >= 1 && !c->prof_on && resident_supported(c, 1, nullptr)) {
+    ASD_CUDA(c, cudaEventRecord(c->ev0, c->stream));
+    asd_status st = launch_resident(c, 1, false, 0x7fffffff);
+    if (st != ASD_OK) return st;
+    ASD_CUDA(c, cudaGetLastError());
+    return finish_run(c, y_out_dev, nullptr, stats_host, launches0, true);
+  }
   int min_a = c->K;
   if (c->n > 0) {
     std::vector<int> a(c->n);
@@ -938,7 +927,7 @@ asd_status asd_sample_host(asd_ctx* ctx, int32_t n_chains, uint64_t chain_id_bas
   if (!y_out_host && n_chains > 0) return fail(c, ASD_ERR_INVALID_ARG, "y_out_host must not be NULL");
   const size_t nd = (size_t)n_chains * c->d;
   // the library's own state / workspace rows serve as staging: y0 -> G (unused until the first
-  // round), cond -> cond_f32 (reset converts it in place)
+  // round), cond -> the drafted-point buffer (reset converts it to bf16 from there)
   const bool need_cond = c->kind == ASD_DEN_RESMLP_BF16 && c->mlp.d_cond > 0;
   if (need_cond && !cond_host && n_chains > 0) return fail(c, ASD_ERR_INVALID_ARG, "cond_host required (d_cond > 0)");
   if (y0_host) ASD_CUDA(c, cudaMemcpyAsync(c->G, y0_host, nd * sizeof(float), cudaMemcpyHostToDevice, c->stream));

@@ -28,7 +28,8 @@ struct RoundCounters {
   unsigned long long rows_total;  // running total of drift evaluations since reset
   unsigned long long rows_verified;  // running total of drift rows the verify kernel read since reset
   int n_eval;                   // chains whose v_a has to be evaluated this round (look-ahead: not all active ones)
-  int pad;
+  int rounds_max;               // written by the finish kernel of a run: max and sum over chains of the round counters
+  unsigned long long rounds_sum;
 };
 
 // Per-step fp32 tables, built on the host in fp64 (asd_create).
@@ -142,7 +143,6 @@ struct Ctx {
   int* rounds = nullptr;     // [max_chains]
   int* wnd = nullptr;        // [max_chains] per-chain speculation length of the next round (adaptive mode)
   int* ema8 = nullptr;       // [max_chains] 8 x running mean of the steps advanced per round (adaptive mode)
-  float* cond_f32 = nullptr; // [max_chains, d_cond]
   int* act = nullptr;        // [max_chains] active position -> chain position
   int* row_off = nullptr;    // [max_chains + 1]
   int* step1 = nullptr;      // [max_chains] cursor of the active chain
@@ -179,6 +179,7 @@ struct Ctx {
   std::map<const void*, int> func_smem;  // kernel -> dynamic shared memory opted in on this context's device
   int gemm_mode = 0;                     // ASD_GEMM_MODE at asd_create: 0 planner, 1 "cta", 2 "pair"
   bool stagger = false;                  // ASD_STAGGER=1 at asd_create
+  int resident_mode = 1;                 // ASD_RESIDENT at asd_create: 0 never, 1 asd_sample / asd_sequential_ddpm, 2 asd_round too
   // One speculation round captured as a CUDA graph per (window, use_u, bound on active chains); replayed
   // on a private stream that is forked from and joined to the caller's stream.
   struct RoundGraph { cudaGraphExec_t exec; long long launches; };
@@ -223,14 +224,22 @@ void launch_pack_appended(Ctx* c, const Lane& L, const int* row_base_dev, int* m
 void launch_pack(Ctx* c, const RowSet& rs);
 void launch_gmm(Ctx* c, const RowSet& rs, float* out);
 void launch_gauss(Ctx* c, const RowSet& rs, float* out);
-void launch_cond_to_bf16(Ctx* c, int n);
-void launch_fill_int(Ctx* c, int* p, int n, int val);
 void launch_traj_seed(Ctx* c);  // trajectory row a_j <- y_j for every chain of the batch
+// asd_reset in one launch: state, cursors, counters, per-chain window state, histogram, trajectory row 0 and the
+// bf16 copy of the conditioning
+void launch_reset(Ctx* c, const float* y0_dev, const float* cond_dev);
+// end of a run in one launch: y -> y_out, rounds -> rounds_out (either may be null), max / sum of the round counters
+void launch_finish(Ctx* c, float* y_out_dev, int* rounds_out_dev);
 
 // ---- MLP forward (asd_gemm.cu) ----------------------------------------------------------
 // Runs the GEMM chain on the rows already packed into mlp.X; writes out[r] for r < *n_rows_dev.
 // pass: 0 = drift at the current points, 1 = drift at the drafted points, 2 = stand-alone call.
 asd_status mlp_forward(Ctx* c, const RowSet& rs, float* out, int pass);
 void launch_wait_selftest(Ctx* c);  // one bounded wait that must run out (failure-path self-test)
+
+// ---- chain-resident round driver for the closed-form drifts (asd_resident.cu) ------------------
+bool resident_supported(const Ctx* c, int window, int* smem_bytes);
+// `max_rounds` iterations of Algorithm 1's while loop for every chain (to the end of the grid if large), one launch
+asd_status launch_resident(Ctx* c, int window, bool use_u, int max_rounds);
 
 }  // namespace asd

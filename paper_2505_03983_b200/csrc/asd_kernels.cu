@@ -7,121 +7,14 @@
 #include <algorithm>
 
 #include "asd_internal.h"
+#include "asd_device.cuh"
 
 namespace asd {
-
-// ---------------------------------------------------------------------------------------------
-// Counter-based randomness (Algorithm 1, "sample u, xi"): Philox4x32-10, counter =
-// (dimension block, step, chain id, tag).
-// ---------------------------------------------------------------------------------------------
-// Round keys of the ten rounds (key + r * Weyl constant), computed once on the host and passed in
-// the kernel arguments, so a round is two 32x32->64 multiplies and two three-input xors.
-struct PhiloxKeys {
-  uint32_t k[20];
-};
-
-PhiloxKeys make_philox_keys(uint64_t seed) {
-  PhiloxKeys K;
-  uint32_t k0 = (uint32_t)(seed & 0xffffffffull), k1 = (uint32_t)(seed >> 32);
-  for (int r = 0; r < 10; ++r) {
-    K.k[2 * r] = k0;
-    K.k[2 * r + 1] = k1;
-    k0 += 0x9E3779B9u;
-    k1 += 0xBB67AE85u;
-  }
-  return K;
-}
-
-__device__ __forceinline__ uint4 philox4x32_10(uint4 c, const PhiloxKeys& K) {
-  constexpr uint32_t M0 = 0xD2511F53u, M1 = 0xCD9E8D57u;
-#pragma unroll
-  for (int r = 0; r < 10; ++r) {
-    const uint64_t p0 = (uint64_t)M0 * c.x;
-    const uint64_t p1 = (uint64_t)M1 * c.z;
-    c = make_uint4((uint32_t)(p1 >> 32) ^ c.y ^ K.k[2 * r], (uint32_t)p1, (uint32_t)(p0 >> 32) ^ c.w ^ K.k[2 * r + 1],
-                   (uint32_t)p0);
-  }
-  return c;
-}
-
-// U(r) = ((r >> 9) + 0.5) 2^-23, exactly: the 23 bits become the mantissa of a float in [1, 2) and
-// the subtraction of 1 - 2^-24 is exact (the result has 24 significant bits).
-__device__ __forceinline__ float uniform_from_word(uint32_t r) {
-  return __uint_as_float((r >> 9) | 0x3f800000u) - 0.99999994f;
-}
-
-// Box-Muller on the special-function unit: radius = sqrt(-2 ln2 lg2 U(r_even)) with lg2.approx and
-// sqrt.approx, angle 2 pi U(r_odd) shifted by -pi into [-pi, pi] (where sin.approx / cos.approx are
-// most accurate); the shift negates both outputs, which the sign of the radius undoes.
-__device__ __forceinline__ void box_muller(uint32_t r_even, uint32_t r_odd, float& n_even, float& n_odd) {
-  float rad;
-  asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(rad) : "f"(-1.3862943611198906f * __log2f(uniform_from_word(r_even))));
-  // 2 pi (f - 1 + 2^-24) - pi with f = 1.mantissa in [1, 2)
-  const float th = fmaf(__uint_as_float((r_odd >> 9) | 0x3f800000u), 6.283185307179586f, -9.424777586315302f);
-  n_even = -rad * __cosf(th);
-  n_odd = -rad * __sinf(th);
-}
-
-// xi_step[4q .. 4q+3]
-__device__ __forceinline__ float4 xi4(uint32_t q, uint32_t step, uint32_t chain, const PhiloxKeys& K) {
-  const uint4 r = philox4x32_10(make_uint4(q, step, chain, 0u), K);
-  float4 n;
-  box_muller(r.x, r.y, n.x, n.y);
-  box_muller(r.z, r.w, n.z, n.w);
-  return n;
-}
-
-// ln u_step: evaluated once per slot, with the accurate logarithm (it decides the accept test).
-__device__ __forceinline__ float ln_u(uint32_t step, uint32_t chain, const PhiloxKeys& K) {
-  const uint4 r = philox4x32_10(make_uint4(0u, step, chain, 1u), K);
-  return logf(uniform_from_word(r.x));
-}
-
-// Loads / stores of the 4 dims of block q with a ragged tail (d not a multiple of 4).
-__device__ __forceinline__ float4 load4(const float* row, int q, int d, bool vec) {
-  if (vec) return *reinterpret_cast<const float4*>(row + 4 * q);
-  float4 r = make_float4(0.f, 0.f, 0.f, 0.f);
-  const int b = 4 * q;
-  if (b + 0 < d) r.x = row[b + 0];
-  if (b + 1 < d) r.y = row[b + 1];
-  if (b + 2 < d) r.z = row[b + 2];
-  if (b + 3 < d) r.w = row[b + 3];
-  return r;
-}
-
-__device__ __forceinline__ void store4(float* row, int q, int d, bool vec, float4 val) {
-  if (vec) {
-    *reinterpret_cast<float4*>(row + 4 * q) = val;
-    return;
-  }
-  const int b = 4 * q;
-  if (b + 0 < d) row[b + 0] = val.x;
-  if (b + 1 < d) row[b + 1] = val.y;
-  if (b + 2 < d) row[b + 2] = val.z;
-  if (b + 3 < d) row[b + 3] = val.w;
-}
-
-// Window of chain j this round: its own speculation length (adaptive mode, kept within 1..window) or
-// the common one, cut at the end of the grid (Algorithm 1: b = min(K, a + theta)).
-__device__ __forceinline__ int chain_window(const int* wnd, int j, int window, int K, int a) {
-  const int theta = wnd ? max(1, min(wnd[j], window)) : window;
-  return min(theta, K - a);
-}
-
-__device__ __forceinline__ float warp_sum(float x) {
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
-  return x;
-}
 
 // ---------------------------------------------------------------------------------------------
 // Round driver bookkeeping: compact the chains with a < K into the active list and lay out the
 // pass-2 rows (exclusive scan of w - 1).  One block; n is at most a few tens of thousands.
 // ---------------------------------------------------------------------------------------------
-// Rows a chain drafts: its window minus the last slot (rebuilt by the verify kernel), plus - with
-// look-ahead - that last slot after all, when there is a step beyond it whose drift it can supply.
-__device__ __forceinline__ int drafted_rows(int w, int a, int K, int la) { return w - 1 + ((la && a + w < K) ? 1 : 0); }
-
 __global__ void __launch_bounds__(1024) prep_kernel(const int* __restrict__ a, const int* __restrict__ wnd, int n, int K,
                                                     int window, const int* __restrict__ has_v, int la,
                                                     int* __restrict__ act, int* __restrict__ row_off,
@@ -513,12 +406,6 @@ struct VerifyArgs {
 
 constexpr int kVerifyMaxWarps = 8;
 
-// ln ratio of Algorithm 3 from the two reductions, with the rounding of every operation spelled out so
-// that every kernel that evaluates it gets the same bits: -(eta/sigma) <xi, delta> - (eta^2 / 2 sigma^2) |delta|^2.
-__device__ __forceinline__ float ln_ratio_of(float c1, float c2, float dot, float nrm) {
-  return __fmaf_rn(-c1, dot, -__fmul_rn(c2, nrm));
-}
-
 __global__ void __launch_bounds__(256) verify_kernel(const VerifyArgs A) {
   __shared__ float s_part[2][kVerifyMaxWarps][2][kVerifyMaxWarps];  // [group parity][slot][dot | nrm][warp of team]
   __shared__ float s_lu[2][kVerifyMaxWarps];                        // [group parity][slot] ln u
@@ -756,30 +643,8 @@ __global__ void __launch_bounds__(128) gmm_kernel(RowSet rs, int d, GmmParams P,
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, wpb = blockDim.x >> 5;
   float* lg = s_logit + warp * P.n_comp;
   const int n_rows = *rs.n_rows_dev;
-  for (int r = blockIdx.x * wpb + warp; r < n_rows; r += gridDim.x * wpb) {
-    const float* y = rs.ysrc + (size_t)(rs.row_map ? rs.row_map[r] : r) * d;
-    const float t = tt[rs.row_step[r]];
-    const float inv_den = 1.f / (1.f + t * P.s2);
-    float mx = -INFINITY;
-    for (int c = 0; c < P.n_comp; ++c) {
-      float dot = 0.f;
-      for (int k = lane; k < d; k += 32) dot = fmaf(y[k], P.means[(size_t)c * d + k], dot);
-      dot = warp_sum(dot);
-      const float l = P.log_pi[c] + (dot - 0.5f * t * P.cnorm[c]) * inv_den;
-      if (lane == 0) lg[c] = l;
-      mx = fmaxf(mx, l);
-    }
-    __syncwarp();
-    float sum = 0.f;
-    for (int c = 0; c < P.n_comp; ++c) sum += expf(lg[c] - mx);
-    const float inv_sum = 1.f / sum;
-    for (int k = lane; k < d; k += 32) {
-      float acc = 0.f;
-      for (int c = 0; c < P.n_comp; ++c) acc = fmaf(expf(lg[c] - mx) * inv_sum, P.means[(size_t)c * d + k], acc);
-      out[(size_t)r * d + k] = (acc + P.s2 * y[k]) * inv_den;
-    }
-    __syncwarp();
-  }
+  for (int r = blockIdx.x * wpb + warp; r < n_rows; r += gridDim.x * wpb)
+    gmm_point(rs.ysrc + (size_t)(rs.row_map ? rs.row_map[r] : r) * d, tt[rs.row_step[r]], d, P, lg, out + (size_t)r * d, lane);
 }
 
 void launch_gmm(Ctx* c, const RowSet& rs, float* out) {
@@ -802,18 +667,9 @@ __global__ void __launch_bounds__(128) gauss_kernel(RowSet rs, int d, GaussParam
     const float t = tt[rs.row_step[r]];
     for (int k = threadIdx.x; k < d; k += blockDim.x) ys[k] = y[k];
     __syncthreads();
-    for (int jj = threadIdx.x; jj < d; jj += blockDim.x) {
-      float z = 0.f;  // (Q^T y)_j
-      for (int i = 0; i < d; ++i) z = fmaf(P.Q[(size_t)i * d + jj], ys[i], z);
-      const float lam = P.lam[jj];
-      ws[jj] = (P.qmu[jj] + lam * z) / (1.f + t * lam);
-    }
+    for (int jj = threadIdx.x; jj < d; jj += blockDim.x) ws[jj] = gauss_coord(P.Q, ys, d, jj, P.qmu[jj], P.lam[jj], t);
     __syncthreads();
-    for (int i = threadIdx.x; i < d; i += blockDim.x) {
-      float m = 0.f;
-      for (int jj = 0; jj < d; ++jj) m = fmaf(P.Qt[(size_t)jj * d + i], ws[jj], m);
-      out[(size_t)r * d + i] = m;
-    }
+    for (int i = threadIdx.x; i < d; i += blockDim.x) out[(size_t)r * d + i] = gauss_out(P.Qt, ws, d, i);
     __syncthreads();
   }
 }
@@ -908,20 +764,6 @@ void launch_pack_appended(Ctx* c, const Lane& L, const int* row_base_dev, int* m
   c->launches++;
 }
 
-__global__ void cond_to_bf16_kernel(const float* __restrict__ src, __nv_bfloat16* __restrict__ dst, size_t n) {
-  for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x)
-    dst[i] = __float2bfloat16_rn(src[i]);
-}
-
-void launch_cond_to_bf16(Ctx* c, int n) {
-  const size_t total = (size_t)n * c->mlp.d_cond;
-  if (total == 0) return;
-  int blocks = (int)((total + 255) / 256);
-  blocks = blocks > 1024 ? 1024 : blocks;
-  cond_to_bf16_kernel<<<blocks, 256, 0, c->stream>>>(c->cond_f32, const_cast<__nv_bfloat16*>(c->mlp.cond), total);
-  c->launches++;
-}
-
 // Trajectory bookkeeping: the state a chain is (re)started from is row a of its trajectory.
 __global__ void traj_seed_kernel(const int* __restrict__ a, const float* __restrict__ y, float* __restrict__ traj, int n,
                                  int K, int d) {
@@ -938,15 +780,128 @@ void launch_traj_seed(Ctx* c) {
   c->launches++;
 }
 
-__global__ void fill_int_kernel(int* p, int n, int val) {
-  for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x) p[i] = val;
+struct ResetArgs {
+  int n, max_chains, d, d_cond, K, hist_len, wnd0, ema0;
+  const float* y0;
+  const float* cond;
+  float* y;
+  int* a;
+  int* rounds;
+  int* acc_len;
+  int* wnd;
+  int* ema8;
+  int* has_v;
+  __nv_bfloat16* cond_bf16;
+  RoundCounters* counters;  // [2]
+  unsigned long long* hist;
+  float* traj;
+};
+
+__global__ void __launch_bounds__(256) reset_kernel(const ResetArgs A) {
+  const size_t tid = blockIdx.x * (size_t)blockDim.x + threadIdx.x, nt = (size_t)gridDim.x * blockDim.x;
+  const size_t nd = (size_t)A.n * A.d;
+  for (size_t e = tid; e < nd; e += nt) {
+    const float v = A.y0 ? A.y0[e] : 0.f;
+    A.y[e] = v;
+    if (A.traj) {
+      const size_t j = e / A.d, k = e - j * A.d;
+      A.traj[j * (size_t)(A.K + 1) * A.d + k] = v;  // row 0 of chain j
+    }
+  }
+  for (size_t j = tid; j < (size_t)A.max_chains; j += nt) {
+    A.a[j] = 0;
+    A.rounds[j] = 0;
+    A.acc_len[j] = -1;
+    A.wnd[j] = A.wnd0;
+    A.ema8[j] = A.ema0;
+    if (A.has_v) A.has_v[j] = 0;
+  }
+  for (size_t e = tid; e < (size_t)A.hist_len; e += nt) A.hist[e] = 0ull;
+  const size_t nc = (size_t)A.n * A.d_cond;
+  for (size_t e = tid; e < nc; e += nt) A.cond_bf16[e] = __float2bfloat16_rn(A.cond[e]);
+  if (tid < 2) {
+    const int err = A.counters[tid].err;  // a pending device error survives until the host has read it
+    RoundCounters z{};
+    z.err = err;
+    A.counters[tid] = z;
+  }
 }
 
-void launch_fill_int(Ctx* c, int* p, int n, int val) {
-  if (n <= 0) return;
-  int blocks = (n + 255) / 256;
-  blocks = blocks > 1024 ? 1024 : blocks;
-  fill_int_kernel<<<blocks, 256, 0, c->stream>>>(p, n, val);
+void launch_reset(Ctx* c, const float* y0_dev, const float* cond_dev) {
+  ResetArgs A{};
+  A.n = c->n;
+  A.max_chains = c->max_chains;
+  A.d = c->d;
+  A.d_cond = (c->kind == ASD_DEN_RESMLP_BF16 && cond_dev) ? c->mlp.d_cond : 0;
+  A.K = c->K;
+  A.hist_len = c->window + 1;
+  A.ema0 = 32;  // adaptive mode starts every chain at 8 x mean = 32, i.e. a speculation length of min(window, 8)
+  A.wnd0 = std::max(2, std::min(c->window, 2 + (3 * A.ema0) / 16));
+  A.y0 = y0_dev;
+  A.cond = cond_dev;
+  A.y = c->y;
+  A.a = c->a;
+  A.rounds = c->rounds;
+  A.acc_len = c->acc_len;
+  A.wnd = c->wnd;
+  A.ema8 = c->ema8;
+  A.has_v = c->has_v;
+  A.cond_bf16 = const_cast<__nv_bfloat16*>(c->mlp.cond);
+  A.counters = c->counters;
+  A.hist = c->hist;
+  A.traj = c->traj;
+  const size_t work = std::max<size_t>((size_t)c->n * c->d, (size_t)c->max_chains);
+  const int blocks = (int)std::min<size_t>((work + 255) / 256, (size_t)8 * c->num_sms);
+  reset_kernel<<<std::max(blocks, 1), 256, 0, c->stream>>>(A);
+  c->launches++;
+}
+
+// End of a run: block 0 reduces the chains' round counters, the others copy the results out.
+__global__ void __launch_bounds__(256) finish_kernel(const float* __restrict__ y, const int* __restrict__ rounds, int n, int d,
+                                                     float* __restrict__ y_out, int* __restrict__ rounds_out,
+                                                     RoundCounters* __restrict__ cnt) {
+  if (blockIdx.x == 0) {
+    __shared__ unsigned long long s_sum[8];
+    __shared__ int s_max[8];
+    unsigned long long sum = 0ull;
+    int mx = 0;
+    for (int j = threadIdx.x; j < n; j += blockDim.x) {
+      const int r = rounds[j];
+      sum += (unsigned long long)r;
+      mx = max(mx, r);
+      if (rounds_out) rounds_out[j] = r;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      sum += __shfl_xor_sync(0xffffffffu, sum, o);
+      mx = max(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    }
+    if ((threadIdx.x & 31) == 0) {
+      s_sum[threadIdx.x >> 5] = sum;
+      s_max[threadIdx.x >> 5] = mx;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      for (int x = 1; x < 8; ++x) {
+        sum += s_sum[x];
+        mx = max(mx, s_max[x]);
+      }
+      cnt->rounds_sum = sum;
+      cnt->rounds_max = mx;
+    }
+    if (gridDim.x > 1) return;
+  }
+  if (!y_out) return;
+  const size_t nd = (size_t)n * d;
+  const size_t b0 = gridDim.x > 1 ? blockIdx.x - 1 : 0, nb = gridDim.x > 1 ? gridDim.x - 1 : 1;
+  for (size_t e = b0 * blockDim.x + threadIdx.x; e < nd; e += nb * blockDim.x) y_out[e] = y[e];
+}
+
+void launch_finish(Ctx* c, float* y_out_dev, int* rounds_out_dev) {
+  const size_t nd = (size_t)c->n * c->d;
+  const int copy_blocks = y_out_dev ? (int)std::min<size_t>((nd + 255) / 256, (size_t)8 * c->num_sms) : 0;
+  finish_kernel<<<1 + (nd > 4096 ? copy_blocks : 0), 256, 0, c->stream>>>(c->y, c->rounds, c->n, c->d, y_out_dev,
+                                                                         rounds_out_dev, c->counters);
   c->launches++;
 }
 

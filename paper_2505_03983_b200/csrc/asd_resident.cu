@@ -1,0 +1,493 @@
+// Chain-resident round driver for the closed-form drifts (Eq. 4: mixture and Gaussian targets).
+//
+// Chains are independent and a round of these drifts is a few thousand flops per window slot, so nothing
+// forces a kernel boundary between the steps of Algorithm 1: ONE block owns ONE chain and runs the while
+// loop to the end of the grid (or for a given number of rounds) inside a single launch - drift at the
+// current point, draft of the window, drift at every drafted point, Verifier (Algorithms 2 and 3),
+// reflection, advance - with the chain's state, its window of noise, drafted points and drifts in shared
+// memory.  Every expression is evaluated in the order of the per-phase kernels (asd_kernels.cu), with the
+// shared device functions of asd_device.cuh, so a run gives the same bits either way.
+#include <algorithm>
+
+#include "asd_device.cuh"
+#include "asd_internal.h"
+
+namespace asd {
+
+namespace {
+
+constexpr int kResThreads = 256;
+constexpr int kResWarps = kResThreads / 32;
+constexpr int kResMaxSmem = 200 * 1024;
+
+struct ResidentArgs {
+  int d, dp, nq, vec, K, window, wcap, use_u, all_slots, max_rounds, n;
+  PhiloxKeys keys;
+  uint64_t chain_base;
+  int* a;
+  int* rounds;
+  float* y;
+  int* wnd;   // per-chain speculation length (adaptive mode), or null
+  int* ema8;
+  Tables tab;
+  GmmParams gmm;
+  GaussParams gauss;
+  int* acc_len;
+  float* dbg_lr;  // diagnostics of the last round run (ASD_FLAG_DEBUG_DUMP), or null
+  float* dbg_lu;
+  int dbg_stride;
+  float* traj;               // [n, K + 1, d], or null
+  unsigned long long* hist;  // [window + 1]
+  RoundCounters* cnt;
+};
+
+// Shared-memory layout in floats; the vector arrays first (rows of dp = 4 nq floats, 16-byte aligned).
+struct ResidentLayout {
+  int y, v, xi, yh, g, lu, dot, nrm, tab, extra, total;
+};
+
+__host__ __device__ inline ResidentLayout resident_layout(int kind, int d, int dp, int wcap, int n_comp) {
+  ResidentLayout L;
+  int o = 0;
+  L.y = o;    o += dp;
+  L.v = o;    o += dp;
+  L.xi = o;   o += wcap * dp;   // xi of slots 1..w
+  L.yh = o;   o += wcap * dp;   // drafted points of slots 1..w-1
+  L.g = o;    o += wcap * dp;   // drift at the drafted points
+  const int wp = (wcap + 4) & ~3;
+  L.lu = o;   o += wp;
+  L.dot = o;  o += wp;
+  L.nrm = o;  o += wp;
+  L.tab = o;  o += 5 * wp;                  // eta, sigma, c1, c2, t of the window's steps
+  L.extra = o;
+  if (kind == ASD_DEN_GAUSS_LINEAR)
+    o += 2 * d * d + 2 * d + wcap * dp;     // Q, Qt, qmu, lam, eigen-coordinates per point (rows of dp)
+  else
+    o += kResWarps * n_comp + n_comp * (d + 2);  // the warps' logits; means, ln pi, |c|^2
+  L.total = o;
+  return L;
+}
+
+// Gaussian posterior mean of n_pts points (rows of dp floats in shared memory) by the whole block.
+// One item = one eigen-coordinate (then one output coordinate) of a group of kPts points: the matrix element is
+// loaded once for the group and the points' sums run side by side, each in the order of dot_strided4 (four
+// interleaved partial sums), so the bits are those of gauss_coord / gauss_out point by point.
+template <int kPts>
+__device__ __forceinline__ void resident_gauss(const ResidentArgs& A, const float* sm, const ResidentLayout& L,
+                                               const float* src, float* dst, int n_pts, const float* s_t) {
+  const int tid = threadIdx.x, d = A.d;
+  const float* sQ = sm + L.extra;
+  const float* sQt = sQ + d * d;
+  const float* s_qmu = sQt + d * d;
+  const float* s_lam = s_qmu + d;
+  float* s_ws = const_cast<float*>(s_lam) + d;
+  const int groups = (n_pts + kPts - 1) / kPts;
+  const int d4 = d & ~3;
+  for (int it = tid; it < groups * d; it += kResThreads) {
+    const int pg = it / d, jj = it - pg * d, p0 = pg * kPts;
+    const int np = min(kPts, n_pts - p0);
+    const float* y0 = src + (size_t)p0 * A.dp;
+    float z[kPts][4];
+#pragma unroll
+    for (int u = 0; u < kPts; ++u) z[u][0] = z[u][1] = z[u][2] = z[u][3] = 0.f;
+#pragma unroll 4
+    for (int i = 0; i < d4; i += 4) {  // four terms per 16-byte (broadcast) load of each point
+      const float q0 = sQ[(size_t)i * d + jj], q1 = sQ[(size_t)(i + 1) * d + jj], q2 = sQ[(size_t)(i + 2) * d + jj],
+                  q3 = sQ[(size_t)(i + 3) * d + jj];
+#pragma unroll
+      for (int u = 0; u < kPts; ++u) {
+        const float4 yv = *reinterpret_cast<const float4*>(y0 + (size_t)min(u, np - 1) * A.dp + i);
+        z[u][0] = fmaf(q0, yv.x, z[u][0]);
+        z[u][1] = fmaf(q1, yv.y, z[u][1]);
+        z[u][2] = fmaf(q2, yv.z, z[u][2]);
+        z[u][3] = fmaf(q3, yv.w, z[u][3]);
+      }
+    }
+#pragma unroll
+    for (int r = 0; r < 3; ++r) {  // the last d mod 4 terms
+      if (d4 + r < d) {
+        const float qv = sQ[(size_t)(d4 + r) * d + jj];
+#pragma unroll
+        for (int u = 0; u < kPts; ++u) z[u][r] = fmaf(qv, y0[(size_t)min(u, np - 1) * A.dp + d4 + r], z[u][r]);
+      }
+    }
+    const float qmu = s_qmu[jj], lam = s_lam[jj];
+#pragma unroll
+    for (int u = 0; u < kPts; ++u)
+      if (u < np) s_ws[(size_t)(p0 + u) * A.dp + jj] = __fdiv_rn(fmaf(lam, sum4(z[u]), qmu), fmaf(s_t[p0 + u], lam, 1.f));
+  }
+  __syncthreads();
+  for (int it = tid; it < groups * d; it += kResThreads) {
+    const int pg = it / d, i = it - pg * d, p0 = pg * kPts;
+    const int np = min(kPts, n_pts - p0);
+    const float* w0 = s_ws + (size_t)p0 * A.dp;
+    float m[kPts][4];
+#pragma unroll
+    for (int u = 0; u < kPts; ++u) m[u][0] = m[u][1] = m[u][2] = m[u][3] = 0.f;
+#pragma unroll 4
+    for (int jj = 0; jj < d4; jj += 4) {
+      const float q0 = sQt[(size_t)jj * d + i], q1 = sQt[(size_t)(jj + 1) * d + i], q2 = sQt[(size_t)(jj + 2) * d + i],
+                  q3 = sQt[(size_t)(jj + 3) * d + i];
+#pragma unroll
+      for (int u = 0; u < kPts; ++u) {
+        const float4 wv = *reinterpret_cast<const float4*>(w0 + (size_t)min(u, np - 1) * A.dp + jj);
+        m[u][0] = fmaf(q0, wv.x, m[u][0]);
+        m[u][1] = fmaf(q1, wv.y, m[u][1]);
+        m[u][2] = fmaf(q2, wv.z, m[u][2]);
+        m[u][3] = fmaf(q3, wv.w, m[u][3]);
+      }
+    }
+#pragma unroll
+    for (int r = 0; r < 3; ++r) {
+      if (d4 + r < d) {
+        const float qv = sQt[(size_t)(d4 + r) * d + i];
+#pragma unroll
+        for (int u = 0; u < kPts; ++u) m[u][r] = fmaf(qv, w0[(size_t)min(u, np - 1) * A.dp + d4 + r], m[u][r]);
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < kPts; ++u)
+      if (u < np) dst[(size_t)(p0 + u) * A.dp + i] = sum4(m[u]);
+  }
+  __syncthreads();
+}
+
+template <int KIND>
+__device__ __forceinline__ void resident_drift(const ResidentArgs& A, const float* sm, const ResidentLayout& L,
+                                               const float* src, float* dst, int n_pts, const float* s_t) {
+  // dst[p] = g(s_t[p], src[p]) for p < n_pts (rows of dp floats; s_t: the points' times); ends with a block barrier
+  if (KIND == ASD_DEN_GMM_ISO) {
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    float* lg = const_cast<float*>(sm) + L.extra + warp * A.gmm.n_comp;
+    GmmParams P = A.gmm;  // the copy in shared memory
+    P.means = sm + L.extra + kResWarps * A.gmm.n_comp;
+    P.log_pi = P.means + (size_t)A.gmm.n_comp * A.d;
+    P.cnorm = P.log_pi + A.gmm.n_comp;
+    for (int p = warp; p < n_pts; p += kResWarps)
+      gmm_point(src + (size_t)p * A.dp, s_t[p], A.d, P, lg, dst + (size_t)p * A.dp, lane);
+    __syncthreads();
+  } else if (n_pts * A.d <= kResThreads) {
+    resident_gauss<1>(A, sm, L, src, dst, n_pts, s_t);  // few points: an item per thread is already all there is
+  } else {
+    resident_gauss<4>(A, sm, L, src, dst, n_pts, s_t);
+  }
+}
+
+template <int KIND>
+__global__ void __launch_bounds__(kResThreads) resident_kernel(const ResidentArgs A) {
+  extern __shared__ float4 smem4[];
+  float* sm = reinterpret_cast<float*>(smem4);
+  __shared__ int s_first[kResWarps];
+  const int j = blockIdx.x;
+  if (j >= A.n) return;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  int a = A.a[j];
+  if (a >= A.K) {
+    if (tid == 0) A.acc_len[j] = -1;
+    return;
+  }
+  const ResidentLayout L = resident_layout(KIND, A.d, A.dp, A.wcap, A.gmm.n_comp);
+  float* sy = sm + L.y;
+  float* sv = sm + L.v;
+  float4* sXi4 = reinterpret_cast<float4*>(sm + L.xi);
+  float4* sYh4 = reinterpret_cast<float4*>(sm + L.yh);
+  float4* sG4 = reinterpret_cast<float4*>(sm + L.g);
+  float* s_lu = sm + L.lu;
+  float* s_dot = sm + L.dot;
+  float* s_nrm = sm + L.nrm;
+  const int wp = (A.wcap + 4) & ~3;
+  float* s_eta = sm + L.tab;   // [k] = eta_{a+k}, k = 0 .. w-1   (step a+k -> a+k+1)
+  float* s_sig = s_eta + wp;   //       sigma_{a+k+1}
+  float* s_c1 = s_sig + wp;
+  float* s_c2 = s_c1 + wp;
+  float* s_t = s_c2 + wp;      // [k] = t_{a+k}, k = 0 .. w
+  const int nq = A.nq, d = A.d;
+  const uint32_t chain = (uint32_t)(A.chain_base + (uint64_t)j);
+
+  // the chain's state, padded with zeros up to dp, and the target's parameters
+  for (int e = tid; e < A.dp; e += kResThreads) {
+    sy[e] = e < d ? A.y[(size_t)j * d + e] : 0.f;
+    sv[e] = 0.f;
+  }
+  if (KIND == ASD_DEN_GAUSS_LINEAR) {
+    float* sQ = sm + L.extra;
+    for (int e = tid; e < d * d; e += kResThreads) {
+      sQ[e] = A.gauss.Q[e];
+      sQ[d * d + e] = A.gauss.Qt[e];
+    }
+    for (int e = tid; e < d; e += kResThreads) {
+      sQ[2 * d * d + e] = A.gauss.qmu[e];
+      sQ[2 * d * d + d + e] = A.gauss.lam[e];
+    }
+  } else {
+    float* sp = sm + L.extra + kResWarps * A.gmm.n_comp;
+    const int nc = A.gmm.n_comp;
+    for (int e = tid; e < nc * d; e += kResThreads) sp[e] = A.gmm.means[e];
+    for (int e = tid; e < nc; e += kResThreads) {
+      sp[nc * d + e] = A.gmm.log_pi[e];
+      sp[nc * d + nc + e] = A.gmm.cnorm[e];
+    }
+  }
+  int theta_next = A.wnd ? A.wnd[j] : A.window, ema8 = A.wnd ? A.ema8[j] : 0;
+  int r_done = 0, n_last = -1, w_first = 0;
+  long long rows_total = 0, rows_ver = 0, adv_total = 0;
+  __syncthreads();
+
+  while (a < A.K && r_done < A.max_rounds) {
+    const int theta = A.wnd ? max(1, min(theta_next, A.window)) : A.window;
+    const int w = min(theta, A.K - a);  // Algorithm 1: b = min(K, a + theta)
+    if (r_done == 0) w_first = w;
+    // the window's per-step tables: one trip to global memory per round, under the noise generation
+    for (int k = tid; k <= w; k += kResThreads) {
+      s_t[k] = A.tab.tt[a + k];
+      if (k < w) {
+        s_eta[k] = A.tab.eta[a + k];
+        s_sig[k] = A.tab.sig[a + k];
+        s_c1[k] = A.tab.c1[a + k];
+        s_c2[k] = A.tab.c2[a + k];
+      }
+    }
+    // ln u and xi of every slot of the window (counter-based: the same values in every round that reaches a step)
+    for (int k = 1 + tid; k <= w; k += kResThreads) s_lu[k] = A.use_u ? ln_u((uint32_t)(a + k), chain, A.keys) : 0.f;
+    for (int it = tid; it < w * nq; it += kResThreads) {
+      const int k = it / nq, q = it - k * nq;
+      sXi4[it] = xi4((uint32_t)q, (uint32_t)(a + k + 1), chain, A.keys);
+    }
+    __syncthreads();
+    // first model call: v_a = g(t_a, y_a)
+    resident_drift<KIND>(A, sm, L, sy, sv, 1, s_t);
+    // draft: y^_{a+k} = y^_{a+k-1} + eta v_a + sigma xi_{a+k}, k = 1 .. w-1
+    if (tid < nq && w > 1) {
+      float4 yh = reinterpret_cast<const float4*>(sy)[tid];
+      const float4 v = reinterpret_cast<const float4*>(sv)[tid];
+      for (int k = 1; k < w; ++k) {
+        const float eta = s_eta[k - 1], sig = s_sig[k - 1];
+        const float4 xi = sXi4[(k - 1) * nq + tid];
+        yh.x = fmaf(sig, xi.x, fmaf(eta, v.x, yh.x));
+        yh.y = fmaf(sig, xi.y, fmaf(eta, v.y, yh.y));
+        yh.z = fmaf(sig, xi.z, fmaf(eta, v.z, yh.z));
+        yh.w = fmaf(sig, xi.w, fmaf(eta, v.w, yh.w));
+        sYh4[(k - 1) * nq + tid] = yh;
+      }
+    }
+    __syncthreads();
+    // second model call: the drift at every drafted prefix point
+    if (w > 1) resident_drift<KIND>(A, sm, L, sm + L.yh, sm + L.g, w - 1, s_t + 1);
+    // Verifier: <xi, delta> and |delta|^2 per slot, one warp per slot, in the reduction order of the verify kernel
+    for (int k = 2 + warp; k <= w; k += kResWarps) {
+      float dot = 0.f, nrm = 0.f;
+      for (int q = lane; q < nq; q += 32) {
+        const float4 vv = reinterpret_cast<const float4*>(sv)[q];
+        const float4 gg = sG4[(k - 2) * nq + q];
+        const float4 xi = sXi4[(k - 1) * nq + q];
+        float4 dl = make_float4(vv.x - gg.x, vv.y - gg.y, vv.z - gg.z, vv.w - gg.w);
+        if (!A.vec) {
+          const int b = 4 * q;
+          if (b + 1 >= d) dl.y = 0.f;
+          if (b + 2 >= d) dl.z = 0.f;
+          if (b + 3 >= d) dl.w = 0.f;
+        }
+        dot = fmaf(xi.x, dl.x, dot);
+        dot = fmaf(xi.y, dl.y, dot);
+        dot = fmaf(xi.z, dl.z, dot);
+        dot = fmaf(xi.w, dl.w, dot);
+        nrm = fmaf(dl.x, dl.x, nrm);
+        nrm = fmaf(dl.y, dl.y, nrm);
+        nrm = fmaf(dl.z, dl.z, nrm);
+        nrm = fmaf(dl.w, dl.w, nrm);
+      }
+      dot = warp_sum(dot);
+      nrm = warp_sum(nrm);
+      if (lane == 0) {
+        // the partial of a one-warp team is added to zero in the verify kernel: x + 0 = x
+        s_dot[k] = dot;
+        s_nrm[k] = nrm;
+      }
+    }
+    __syncthreads();
+    // first rejected slot
+    int first = w + 1;
+    for (int k = 2 + tid; k <= w; k += kResThreads) {
+      const float lr = ln_ratio_of(s_c1[k - 1], s_c2[k - 1], s_dot[k], s_nrm[k]);
+      const bool acc = (s_lu[k] <= fminf(0.f, lr)) || (s_nrm[k] == 0.f);
+      if (!acc) {
+        first = k;
+        break;
+      }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) first = min(first, __shfl_xor_sync(0xffffffffu, first, o));
+    if (lane == 0) s_first[warp] = first;
+    __syncthreads();
+#pragma unroll
+    for (int x = 0; x < kResWarps; ++x) first = min(first, s_first[x]);
+    const int n = first <= w ? first - 1 : w;  // accepted prefix length
+    const int adv = n < w ? n + 1 : w;
+    if (A.dbg_lr) {
+      for (int k = 1 + tid; k <= w; k += kResThreads) {
+        A.dbg_lu[(size_t)j * A.dbg_stride + k - 1] = s_lu[k];
+        A.dbg_lr[(size_t)j * A.dbg_stride + k - 1] = k == 1 ? 0.f : ln_ratio_of(s_c1[k - 1], s_c2[k - 1], s_dot[k], s_nrm[k]);
+      }
+    }
+    // new state
+    float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (tid < nq) {
+      const float4 v = reinterpret_cast<const float4*>(sv)[tid];
+      if (n < w) {
+        const float eta = s_eta[n], sig = s_sig[n];
+        const float coef = 2.f * s_dot[n + 1] / s_nrm[n + 1];
+        const float4 b = sYh4[(n - 1) * nq + tid];  // n >= 1 always (Lemma 1)
+        const float4 g = sG4[(n - 1) * nq + tid];
+        const float4 xi = sXi4[n * nq + tid];
+        o.x = fmaf(sig, fmaf(-coef, v.x - g.x, xi.x), fmaf(eta, g.x, b.x));
+        o.y = fmaf(sig, fmaf(-coef, v.y - g.y, xi.y), fmaf(eta, g.y, b.y));
+        o.z = fmaf(sig, fmaf(-coef, v.z - g.z, xi.z), fmaf(eta, g.z, b.z));
+        o.w = fmaf(sig, fmaf(-coef, v.w - g.w, xi.w), fmaf(eta, g.w, b.w));
+      } else {
+        const float eta = s_eta[w - 1], sig = s_sig[w - 1];
+        const float4 b = (w == 1) ? reinterpret_cast<const float4*>(sy)[tid] : sYh4[(w - 2) * nq + tid];
+        const float4 xi = sXi4[(w - 1) * nq + tid];
+        o.x = fmaf(sig, xi.x, fmaf(eta, v.x, b.x));
+        o.y = fmaf(sig, xi.y, fmaf(eta, v.y, b.y));
+        o.z = fmaf(sig, xi.z, fmaf(eta, v.z, b.z));
+        o.w = fmaf(sig, xi.w, fmaf(eta, v.w, b.w));
+      }
+      if (!A.vec) {  // keep the padding at zero
+        const int b0 = 4 * tid;
+        if (b0 + 1 >= d) o.y = 0.f;
+        if (b0 + 2 >= d) o.z = 0.f;
+        if (b0 + 3 >= d) o.w = 0.f;
+      }
+    }
+    __syncthreads();  // every reader of the old state is done
+    if (tid < nq) reinterpret_cast<float4*>(sy)[tid] = o;
+    __syncthreads();
+    if (A.traj) {
+      float* tbase = A.traj + ((size_t)j * (A.K + 1) + a) * d;
+      for (int k = 1; k <= adv; ++k) {
+        const float* src = (k < adv) ? sm + L.yh + (size_t)(k - 1) * A.dp : sy;
+        for (int e = tid; e < d; e += kResThreads) tbase[(size_t)k * d + e] = src[e];
+      }
+    }
+    // statistics, in the terms of the per-phase kernels: drift rows made, and drift rows the verify kernel would
+    // have read (it walks the slots in groups and stops after the group with the first rejection)
+    if (tid == 0) {
+      rows_total += w;
+      const int S = kResWarps;
+      int rr = 0;
+      if (w >= 2) rr = (n == w || A.all_slots) ? w - 1 : min(2 + ((n + 1 - 2) / S) * S + S - 1, w) - 1;
+      rows_ver += rr;
+      adv_total += adv;
+      if (A.hist) atomicAdd(&A.hist[n], 1ull);
+    }
+    if (A.wnd) {
+      ema8 = (ema8 + 8 * adv) >> 1;
+      theta_next = max(2, min(A.window, 2 + (3 * ema8) / 16));
+    }
+    a += adv;
+    n_last = n;
+    ++r_done;
+  }
+
+  for (int e = tid; e < d; e += kResThreads) A.y[(size_t)j * d + e] = sy[e];
+  if (tid == 0) {
+    A.a[j] = a;
+    A.rounds[j] += r_done;
+    A.acc_len[j] = n_last;
+    if (A.wnd) {
+      A.wnd[j] = theta_next;
+      A.ema8[j] = ema8;
+    }
+    atomicAdd(&A.cnt->n_active, 1);
+    atomicAdd(&A.cnt->n_eval, 1);
+    atomicAdd(&A.cnt->rows2, w_first - 1);
+    atomicAdd(&A.cnt->accepted, (unsigned long long)adv_total);
+    atomicAdd(&A.cnt->rows_total, (unsigned long long)rows_total);
+    atomicAdd(&A.cnt->rows_verified, (unsigned long long)rows_ver);
+    if (a < A.K) atomicAdd(&A.cnt->n_active_after, 1);
+  }
+}
+
+// The per-call counters start at zero; the running totals and the error word stay.
+__global__ void resident_begin_kernel(RoundCounters* cnt) {
+  cnt->n_active = 0;
+  cnt->rows2 = 0;
+  cnt->n_active_after = 0;
+  cnt->n_eval = 0;
+  cnt->accepted = 0ull;
+}
+
+}  // namespace
+
+// Whether the chain-resident kernel can serve this context (closed-form drift, one-warp reduction teams,
+// the window's working set fits shared memory); *smem_bytes receives the dynamic shared memory it needs.
+bool resident_supported(const Ctx* c, int window, int* smem_bytes) {
+  if (c->kind != ASD_DEN_GMM_ISO && c->kind != ASD_DEN_GAUSS_LINEAR) return false;
+  if (c->lookahead) return false;
+  const int nq = (c->d + 3) / 4;
+  if (nq >= 512 || nq > kResThreads) return false;
+  const ResidentLayout L = resident_layout(c->kind, c->d, 4 * nq, std::max(window, 1), c->gmm.n_comp);
+  const long long bytes = (long long)L.total * 4;
+  if (bytes > kResMaxSmem) return false;
+  if (smem_bytes) *smem_bytes = (int)bytes;
+  return true;
+}
+
+// `max_rounds` iterations of Algorithm 1's while loop (or to the end of the grid) for every chain, one launch.
+asd_status launch_resident(Ctx* c, int window, bool use_u, int max_rounds) {
+  int smem = 0;
+  if (!resident_supported(c, window, &smem)) return ASD_ERR_UNSUPPORTED;
+  if (c->n <= 0) return ASD_OK;
+  ResidentArgs A{};
+  A.d = c->d;
+  A.nq = (c->d + 3) / 4;
+  A.dp = 4 * A.nq;
+  A.vec = (c->d % 4 == 0);
+  A.K = c->K;
+  A.window = window;
+  A.wcap = std::max(window, 1);
+  A.use_u = use_u ? 1 : 0;
+  A.all_slots = c->debug_all_slots ? 1 : 0;
+  A.max_rounds = max_rounds;
+  A.n = c->n;
+  A.keys = make_philox_keys(c->seed);
+  A.chain_base = c->chain_base;
+  A.a = c->a;
+  A.rounds = c->rounds;
+  A.y = c->y;
+  const bool adaptive = c->adaptive && window > 1;
+  A.wnd = adaptive ? c->wnd : nullptr;
+  A.ema8 = c->ema8;
+  A.tab = c->tab;
+  A.gmm = c->gmm;
+  A.gauss = c->gauss;
+  A.acc_len = c->acc_len;
+  A.dbg_lr = c->dbg_lr;
+  A.dbg_lu = c->dbg_lu;
+  A.dbg_stride = c->window;
+  A.traj = c->traj;
+  A.hist = c->hist;
+  A.cnt = c->counters;
+  if (max_rounds < 0x7fffffff) {  // a call that reports per-round counters (asd_round) starts them at zero
+    resident_begin_kernel<<<1, 1, 0, c->stream>>>(c->counters);
+    c->launches++;
+  }
+  const void* fn = c->kind == ASD_DEN_GMM_ISO ? reinterpret_cast<const void*>(&resident_kernel<ASD_DEN_GMM_ISO>)
+                                              : reinterpret_cast<const void*>(&resident_kernel<ASD_DEN_GAUSS_LINEAR>);
+  int& have = c->func_smem[fn];
+  if (smem > have) {
+    if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) {
+      c->err = "resident kernel: shared-memory opt-in failed";
+      return ASD_ERR_CUDA;
+    }
+    have = smem;
+  }
+  if (c->kind == ASD_DEN_GMM_ISO)
+    resident_kernel<ASD_DEN_GMM_ISO><<<c->n, kResThreads, smem, c->stream>>>(A);
+  else
+    resident_kernel<ASD_DEN_GAUSS_LINEAR><<<c->n, kResThreads, smem, c->stream>>>(A);
+  c->launches++;
+  return ASD_OK;
+}
+
+}  // namespace asd

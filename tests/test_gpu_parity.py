@@ -814,3 +814,58 @@ def test_context_created_on_a_busy_side_stream():
             side.synchronize()
     torch.cuda.synchronize()
     assert torch.equal(out, ref) and torch.equal(y1, y_ref) and torch.equal(r1, r_ref)
+
+# ------------------------------------------------------------------ chain-resident kernel (closed-form drifts)
+@pytest.mark.parametrize("name,chains,kw", [("cfg1_gmm2d", 16, {}), ("cfg2_gauss64", 40, {"K": 300}), ("gmm_odd", 9, {}),
+                                            ("gauss_small", 11, {}), ("cfg1_gmm2d", 7, {"K": 200, "window": 200}),
+                                            ("gauss_small", 3, {"window": 1})])
+@pytest.mark.parametrize("flags", ["plain", "adaptive", "all_slots"])
+def test_resident_kernel_equals_per_phase_kernels(name, chains, kw, flags, monkeypatch):
+    """asd_sample / asd_sequential_ddpm on the closed-form drifts run Algorithm 1's while loop inside one launch
+    (a block per chain).  Same expressions in the same order as the per-phase kernels, so with ASD_RESIDENT=0
+    (per-phase kernels, rounds replayed as CUDA graphs) every chain ends in the same bits after the same
+    rounds, with the same row statistics, prefix histogram and trajectory."""
+    from paper_2505_03983_b200.binding import FLAG_ADAPTIVE_WINDOW, FLAG_DEBUG_ALL_SLOTS, FLAG_TRAJECTORY
+    fl = FLAG_TRAJECTORY | {"plain": 0, "adaptive": FLAG_ADAPTIVE_WINDOW, "all_slots": FLAG_DEBUG_ALL_SLOTS}[flags]
+    wl = workloads.make(name, chains=chains, **kw)
+    out = {}
+    for mode in ("0", "1"):
+        monkeypatch.setenv("ASD_RESIDENT", mode)
+        with _sampler(wl, dump=False, flags=fl) as s:
+            s.reset(chains, 90)
+            y, r, st = s.sample()
+            hist, traj = s.prefix_histogram(), s.get_trajectory()
+            wstate = s.get_window_state()
+            s.reset(chains, 90)
+            y_seq, st_seq = s.sequential_ddpm()
+            # stop after a few rounds, resume to the end: the same chain state either way
+            s.reset(chains, 90)
+            for _ in range(3):
+                s.round(want_stats=False)
+            y_res, r_res, _ = s.sample()
+        out[mode] = (y, r, st, hist, traj, wstate, y_seq, st_seq, y_res, r_res)
+    (y0, r0, st0, h0, t0, w0, q0, sq0, yr0, rr0), (y1, r1, st1, h1, t1, w1, q1, sq1, yr1, rr1) = out["0"], out["1"]
+    assert st1.launches <= 2 < st0.launches
+    assert torch.equal(r0, r1) and torch.equal(y0, y1)
+    assert st0.rows_total == st1.rows_total and st0.rows_verified == st1.rows_verified
+    assert st0.rounds_max == st1.rounds_max and st0.rounds_mean == st1.rounds_mean
+    assert np.array_equal(h0, h1) and torch.equal(t0, t1)
+    assert torch.equal(w0[0], w1[0]) and torch.equal(w0[1], w1[1])
+    assert torch.equal(q0, q1) and sq0.rows_total == sq1.rows_total == chains * wl.K
+    assert torch.equal(yr0, yr1) and torch.equal(rr0, rr1) and torch.equal(yr1, y1)
+
+
+@pytest.mark.parametrize("name,chains,rounds,kw", [("cfg1_gmm2d", 16, 60, {}), ("gmm_odd", 9, 30, {}), ("gauss_small", 11, 40, {}),
+                                                   ("cfg2_gauss64", 24, 12, {}), ("cfg1_gmm2d", 5, 12, {"K": 300, "window": 300})])
+@pytest.mark.parametrize("adaptive", [False, True])
+def test_lockstep_resident_kernel_rounds(name, chains, rounds, kw, adaptive, monkeypatch):
+    """The chain-resident kernel limited to one round per launch (ASD_RESIDENT=2 routes asd_round through it),
+    round by round against the oracle like the per-phase kernels."""
+    from paper_2505_03983_b200.binding import FLAG_ADAPTIVE_WINDOW
+    monkeypatch.setenv("ASD_RESIDENT", "2")
+    wl = workloads.make(name, chains=chains, **kw)
+    with _sampler(wl, flags=FLAG_ADAPTIVE_WINDOW if adaptive else 0) as s:
+        worst = lockstep(s, wl, chains, rounds, chain_base=1000, log=_log, adaptive=adaptive)
+        st = s.round()
+        assert st.rows_pass1 == st.n_active_before
+    assert worst["decided"] > 0
