@@ -31,8 +31,8 @@ import workloads  # noqa: E402
 
 DEFAULT_WORKLOAD = "sweep_b512_w64"   # cfg-4 denoiser, 512 chains x window 64, K = 1000 (largest cell)
 # dram__bytes_read.sum + dram__bytes_write.sum of one pass-2 hidden-layer launch of gemm_pair_kernel<256, EPI_HID>
-# at full row count, from the ncu capture summarised in profiles/gemm_pair_hidden_sweep_b512_w16.md; set an entry to
-# None when that kernel changes until the counters are taken again
+# at full row count, from one ncu capture of that kernel; set an entry to None when the kernel changes, until the
+# counters are taken again
 NCU_TRAFFIC_BYTES_PER_LAUNCH = {"sweep_b512_w64": 391_901_184 + 244_783_872}
 METRIC = "samples_per_sec"
 UNIT = "samples/s"
@@ -129,6 +129,76 @@ def oracle_sample_rate(wl, budget_s: float, max_rounds: int):
                        f"(an unfinished chain counts by its fraction of the K steps)")
 
 
+def blas_threads():
+    try:
+        import threadpoolctl
+        info = threadpoolctl.threadpool_info()
+        return max(int(i.get("num_threads", 1)) for i in info) if info else 1
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def oracle_rates(wl, budget_s):
+    """The oracle as it stands on all host cores the BLAS uses, and limited to one thread."""
+    rate, desc = oracle_sample_rate(wl, budget_s, 10 ** 9)
+    out = {"value": rate, "unit": UNIT, "cores": blas_threads(), "kind": "oracle", "sample": desc}
+    try:
+        import threadpoolctl
+        with threadpoolctl.threadpool_limits(limits=1):
+            r1, d1 = oracle_sample_rate(wl, 0.5 * budget_s, 10 ** 9)
+        out["one_core"] = {"value": r1, "unit": UNIT, "cores": 1, "sample": d1}
+    except Exception as e:  # pragma: no cover
+        out["one_core"] = {"unavailable": repr(e)}
+    return out
+
+
+def compact_config(torch, AsdSampler, wl, peaks, steps=3):
+    """One named configuration in brief, on the library's default path (no per-phase events): samples/s, rounds
+    per sample, the sequential sampler on the same GPU, and - from a separate pass with the phase events on - the
+    share of the time spent in the dominant kernel and its roofline fraction."""
+    cond = torch.as_tensor(wl.cond, device="cuda") if wl.kind == "mlp" and wl.d_cond else None
+    n = wl.chains
+    out = {"chains": n, "K": wl.K, "window": wl.window, "d": wl.d}
+    with AsdSampler(wl) as s:
+        for _ in range(3):
+            s.reset(n, 0, cond=cond); s.sample()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(steps):
+            s.reset(n, 0, cond=cond); _, _, st = s.sample()
+        e1.record(); torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / steps
+        out.update(samples_per_sec=n / (ms / 1e3), ms_per_step=ms, rounds_per_sample=st.rounds_mean,
+                   K_over_rounds=wl.K / max(st.rounds_mean, 1e-9), drift_rows_per_sample_over_K=st.rows_total / (n * wl.K),
+                   launches_per_step=st.launches)
+        s.reset(n, 0, cond=cond); s.sequential_ddpm()
+        s.reset(n, 0, cond=cond); _, sq = s.sequential_ddpm()
+        out["sequential_gpu_samples_per_sec"] = n / (sq.ms_total / 1e3)
+        out["wallclock_speedup_asd"] = sq.ms_total / ms
+        s.set_profiling(True)
+        s.reset(n, 0, cond=cond); _, _, stp = s.sample()
+        prof = s.get_profile()
+        s.set_profiling(False)
+    total = sum(v["ms"] for v in prof.values()) or 1.0
+    if wl.kind == "mlp":
+        hid = prof["pass2_gemm_hidden"]
+        flops = 2.0 * wl.width * wl.width * hid["rows"] * wl.n_layers
+        tf = flops / (hid["ms"] / 1e3) / 1e12 if hid["ms"] > 0 else 0.0
+        rows_per_launch = hid["rows"] * wl.n_layers / max(hid["launches"], 1)
+        out["dominant_kernel"] = {"phase": "pass2_gemm_hidden", "share_of_phase_time": hid["ms"] / total,
+                                  "rows_per_launch": rows_per_launch, "tflops": tf,
+                                  "frac_of_sustained_bf16": tf / peaks["bf16_tflops_sustained"],
+                                  "weight_stream_gbs": 2.0 * wl.width * wl.width * hid["launches"] / (hid["ms"] / 1e3) / 1e9
+                                  if hid["ms"] > 0 else 0.0}
+    else:
+        name, v = max(prof.items(), key=lambda kv: kv[1]["ms"])
+        out["dominant_kernel"] = {"phase": name, "share_of_phase_time": v["ms"] / total,
+                                  "note": "per-phase kernels (the timed default path is the chain-resident kernel: "
+                                          "one launch per run, latency-bound on a few thousand flops per slot)"}
+    return out
+
+
 def config_of(wl):
     return {"workload": wl.name, "chains_per_gpu": wl.chains, "K": wl.K, "window": wl.window, "d": wl.d,
             "denoiser": wl.kind, "width": wl.width, "layers": wl.n_layers,
@@ -141,11 +211,7 @@ def run_reference(args):
     if rank != 0:
         return
     wl = workloads.make(args.workload)
-    try:
-        import threadpoolctl
-        cores = max(int(i.get("num_threads", 1)) for i in threadpoolctl.threadpool_info()) if threadpoolctl.threadpool_info() else 1
-    except Exception:
-        cores = os.cpu_count() or 1
+    cores = blas_threads()
     for _ in range(args.warmup):
         oracle_sample_rate(wl, 2.0, 1)
     t0 = time.perf_counter()
@@ -201,7 +267,11 @@ def run_ours(args):
     for _ in range(max(args.warmup, 0)):
         step()
     # ---- timed region: device-resident inputs ------------------------------------------------
-    s.set_profiling(True)
+    # The network workloads are timed with the per-phase events on (the roofline of the dominant kernel is taken
+    # over exactly this region).  The closed-form workloads are timed on the library's default path, the
+    # chain-resident kernel, which has no phases; their per-phase kernels are timed in the second region below.
+    phases_in_main = wl.kind == "mlp"
+    s.set_profiling(phases_in_main)
     clocks = ClockSampler(local)
     barrier()
     clocks.start()
@@ -217,10 +287,12 @@ def run_ours(args):
     barrier()
     clk = clocks.stop()
     ms = ev0.elapsed_time(ev1)
-    prof = s.get_profile()
-    s.set_profiling(False)
-    # ---- the same steps without the per-phase event records (they cost a few microseconds per phase,
-    # which shows in the launch-bound workloads only) -------------------------------------------
+    if phases_in_main:
+        prof = s.get_profile()
+    s.set_profiling(not phases_in_main)
+    # ---- the same steps with the phase events the other way round (off for the network workloads: the events
+    # cost a few microseconds per phase, which shows in the launch-bound workloads only; on for the closed-form
+    # ones: the per-phase kernels instead of the chain-resident one) --------------------------------
     barrier()
     u0, u1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     u0.record()
@@ -229,6 +301,9 @@ def run_ours(args):
     u1.record()
     barrier()
     ms_plain = u0.elapsed_time(u1)
+    if not phases_in_main:
+        prof = s.get_profile()
+    s.set_profiling(False)
     # ---- end to end through the host-buffer entry point -------------------------------------------
     y0_h = torch.zeros((n, wl.d), dtype=torch.float32).pin_memory().numpy()
     cond_h = None if cond is None else torch.as_tensor(cond).pin_memory().numpy()
@@ -310,7 +385,8 @@ def run_ours(args):
                 "d2h_bytes_per_step": int(y_h.nbytes + r_h.nbytes)},
         "sequential_gpu": {"value": n * world / (ms_seq / 1e3), "unit": UNIT, "ms": ms_seq,
                            "wallclock_speedup_asd": (ms_seq) / (ms / args.steps)},
-        "without_phase_events": {"value": total / (ms_plain / 1e3), "unit": UNIT, "ms_per_step": ms_plain / args.steps},
+        ("without_phase_events" if phases_in_main else "per_phase_kernels_with_events"):
+            {"value": total / (ms_plain / 1e3), "unit": UNIT, "ms_per_step": ms_plain / args.steps},
         "adaptive_window": {"value": total / (ms_adapt / 1e3), "unit": UNIT, "ms_per_step": ms_adapt / args.steps,
                             "rounds_per_sample": ad_rounds,
                             "drift_rows_per_sample_over_K": ad_rows / (args.steps * n * wl.K),
@@ -382,23 +458,31 @@ def run_ours(args):
                                            "3 rows per chain-round; bound by instruction issue (Philox + Box-Muller per "
                                            "element) and by the longest accepted prefix, not by HBM"}
     else:
-        ver = prof["verify"]
+        ver = prof["verify"]  # per-phase kernels, second region: the same chains, the same rounds as the first
         vbytes = 4.0 * wl.d * (rows_ver + 3 * ver["rows"])
         vach = vbytes / (ver["ms"] / 1e3) / 1e9 if ver["ms"] > 0 else 0.0
         line["roofline"] = {"kernel": "verify_kernel", "bound": "hbm", "achieved": vach, "peak": peaks["hbm_gbs"],
                             "unit": "GB/s", "frac": vach / peaks["hbm_gbs"], "peak_source": peaks["source"],
                             "launches": ver["launches"], "avg_launch_ms": ver["ms"] / max(ver["launches"], 1),
-                            "traffic": None}
+                            "traffic": None,
+                            "note": "the per-phase verify kernel, timed in the second region; at this size it is bound "
+                                    "by launch latency, and the default path (value) does not launch it at all"}
     # ---- CPU oracle on a bounded sample (rank 0, N = 1 only) -----------------------------------
     if world == 1 and not args.no_cpu_baseline:
-        rate, desc = oracle_sample_rate(wl, 20.0, 10 ** 9)
-        try:
-            import threadpoolctl
-            info = threadpoolctl.threadpool_info()
-            cores = max(int(i.get("num_threads", 1)) for i in info) if info else 1
-        except Exception:
-            cores = os.cpu_count() or 1
-        line["cpu_baseline"] = {"value": rate, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc}
+        line["cpu_baseline"] = oracle_rates(wl, 20.0)
+    # ---- every named configuration in brief (N = 1 only; each costs well under a second of GPU time) ----
+    if world == 1 and not args.no_configs:
+        import dataclasses
+        cfgs = {}
+        for name in ("cfg1_gmm2d", "cfg2_gauss64", "cfg3_policy", "cfg4_image"):
+            if name == wl.name:
+                continue
+            if name == "cfg4_image" and wl.kind == "mlp" and wl.width == 4096 and wl.n_layers == 6 and wl.K == 1000:
+                w4 = dataclasses.replace(wl, name=name, window=32, chains=32)   # the same seeded weights
+            else:
+                w4 = workloads.make(name)
+            cfgs[name] = compact_config(torch, AsdSampler, w4, peaks)
+        line["configs"] = cfgs
     print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()
@@ -412,6 +496,7 @@ def main():
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-configs", action="store_true", help="skip the brief block on the other named configurations")
     ap.add_argument("--sweep", action="store_true",
                     help="run the 12 cells of the batch x window sweep on the cfg-4 denoiser, one JSON line per cell")
     ap.add_argument("--profile-rounds", type=int, default=0,
@@ -432,7 +517,7 @@ def main():
                                              "accepted": st.accepted_total}}))
     elif args.sweep:
         for b, w in workloads.SWEEP_CELLS:
-            args.workload, args.no_cpu_baseline = f"sweep_b{b}_w{w}", True
+            args.workload, args.no_cpu_baseline, args.no_configs = f"sweep_b{b}_w{w}", True, True
             run_ours(args)
     elif args.impl == "reference":
         run_reference(args)
