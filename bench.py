@@ -354,7 +354,19 @@ def run_ours(args):
         sx.close()
         return x0.elapsed_time(x1), float(np.mean(rnds)), nrows
 
+    def phase_shares(flags):
+        """One step on a sampler created with `flags` with the per-phase events on: {phase: share of the summed phase time}."""
+        sx = AsdSampler(wl, flags=flags)
+        sx.reset(n, base, cond=cond_dev); sx.sample()
+        sx.set_profiling(True)
+        sx.reset(n, base, cond=cond_dev); sx.sample()
+        pr = sx.get_profile()
+        sx.close()
+        tot = sum(v["ms"] for v in pr.values()) or 1.0
+        return {k: round(v["ms"] / tot, 4) for k, v in pr.items() if v["launches"]}
+
     ms_adapt, ad_rounds, ad_rows = timed_variant(FLAG_ADAPTIVE_WINDOW)
+    ad_shares = phase_shares(FLAG_ADAPTIVE_WINDOW)
     ms_la, la_rounds, la_rows = timed_variant(FLAG_LOOKAHEAD)
     ms_ala, ala_rounds, ala_rows = timed_variant(FLAG_ADAPTIVE_WINDOW | FLAG_LOOKAHEAD)
 
@@ -390,6 +402,7 @@ def run_ours(args):
         "adaptive_window": {"value": total / (ms_adapt / 1e3), "unit": UNIT, "ms_per_step": ms_adapt / args.steps,
                             "rounds_per_sample": ad_rounds,
                             "drift_rows_per_sample_over_K": ad_rows / (args.steps * n * wl.K),
+                            "phase_time_shares": ad_shares,
                             "note": "same workload, every chain picks its speculation length in 2..window from its "
                                     "own acceptance history (ASD_FLAG_ADAPTIVE_WINDOW); CUDA-graph rounds"},
         "lookahead": {"value": total / (ms_la / 1e3), "unit": UNIT, "ms_per_step": ms_la / args.steps,

@@ -546,6 +546,8 @@ asd_status asd_create(const asd_config* cfg, void* cuda_stream, asd_ctx** out) {
     c->gemm_mode = !gm ? 0 : (!strcmp(gm, "cta") ? 1 : (!strcmp(gm, "pair") ? 2 : 0));
     const char* sg = getenv("ASD_STAGGER");
     c->stagger = sg && sg[0] == '1';
+    const char* vh = getenv("ASD_VERIFY_HORIZON");  // tuning aid: slots verified for all chains at once (default: per launch)
+    c->verify_horizon = vh ? atoi(vh) : -1;
     const char* rm = getenv("ASD_RESIDENT");  // tuning aid: "0" keeps the closed-form drifts on the per-phase kernels
     c->resident_mode = !rm ? 1 : (rm[0] == '0' ? 0 : (rm[0] == '2' ? 2 : 1));
     if (cudaStreamCreateWithFlags(&c->gstream, cudaStreamNonBlocking) != cudaSuccess ||
@@ -610,6 +612,10 @@ asd_status asd_create(const asd_config* cfg, void* cuda_stream, asd_ctx** out) {
     TRY(dev_alloc(c, &c->dbg_lu, n * c->window));
   }
   TRY(dev_alloc(c, &c->acc_len, n));
+  TRY(dev_alloc(c, &c->slot_dot, n * c->window));
+  TRY(dev_alloc(c, &c->slot_nrm, n * c->window));
+  TRY(dev_alloc(c, &c->slot_lu, n * c->window));
+  TRY(dev_alloc(c, &c->first_rej, n));
   TRY(dev_alloc(c, &c->hist, (size_t)c->window + 1));
   if (cfg->flags & ASD_FLAG_TRAJECTORY) TRY(dev_alloc(c, &c->traj, n * ((size_t)K + 1) * d));
   if (c->lookahead) {

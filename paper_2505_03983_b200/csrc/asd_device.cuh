@@ -53,12 +53,16 @@ __device__ __forceinline__ float uniform_from_word(uint32_t r) {
 // sqrt.approx, angle 2 pi U(r_odd) shifted by -pi into [-pi, pi] (where sin.approx / cos.approx are
 // most accurate); the shift negates both outputs, which the sign of the radius undoes.
 __device__ __forceinline__ void box_muller(uint32_t r_even, uint32_t r_odd, float& n_even, float& n_odd) {
-  float rad;
-  asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(rad) : "f"(-1.3862943611198906f * __log2f(uniform_from_word(r_even))));
+  // the uniform is at least 2^-24, never denormal: the flush-to-zero forms need no range fix-up around them
+  float lg, rad, sn, cs;
+  asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(lg) : "f"(uniform_from_word(r_even)));
+  asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(rad) : "f"(-1.3862943611198906f * lg));
   // 2 pi (f - 1 + 2^-24) - pi with f = 1.mantissa in [1, 2)
   const float th = fmaf(__uint_as_float((r_odd >> 9) | 0x3f800000u), 6.283185307179586f, -9.424777586315302f);
-  n_even = -rad * __cosf(th);
-  n_odd = -rad * __sinf(th);
+  asm("cos.approx.ftz.f32 %0, %1;" : "=f"(cs) : "f"(th));
+  asm("sin.approx.ftz.f32 %0, %1;" : "=f"(sn) : "f"(th));
+  n_even = -rad * cs;
+  n_odd = -rad * sn;
 }
 
 // xi_step[4q .. 4q+3]

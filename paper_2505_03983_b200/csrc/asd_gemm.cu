@@ -387,10 +387,11 @@ constexpr int kEpiAhead = (EPI == EPI_OUT) ? 2 : 3;
 // Epilogue of one accumulator tile row: this thread owns output row `row` (tensor-memory lane) and walks
 // its BN columns in chunks of 32.  tcgen05.ld is warp-collective, so every lane runs the loop and only
 // the global accesses are predicated on row_ok.
-template <int EPI, int BN>
+template <int EPI, int BN, bool kAllowFull = true>
 __device__ __forceinline__ void epilogue_tile(const GemmArgs& g, uint32_t taddr0, int row, bool row_ok, int n0, float cs,
                                               float co, const float* ysrc_row) {
-  const bool full_vec =
+  // kAllowFull = false: the caller serves full tiles itself and only ragged ones come here
+  const bool full_vec = kAllowFull &&
       (n0 + BN <= g.n_out) && (EPI == EPI_OUT ? (g.n_out % 4 == 0) : (g.ld_h % 8 == 0));  // warp-uniform
   if (full_vec) {
     constexpr int D = kEpiAhead<EPI>;  // chunks whose operand is in flight ahead of the arithmetic
@@ -416,6 +417,97 @@ __device__ __forceinline__ void epilogue_tile(const GemmArgs& g, uint32_t taddr0
       if (row_ok && col0 < g.n_out) epilogue_chunk<EPI>(g, row, col0, r, cs, co, ysrc_row);
     }
   }
+}
+
+// Epilogue of a 32-row x COLS-column accumulator block by one warp, bf16 outputs (EPI_IN, EPI_HID), with the
+// global accesses staged through shared memory.  tcgen05.ld hands lane l the accumulator ROW l, so a lane reading
+// its residual and writing its output directly touches 32 different rows per instruction (32 memory lines for
+// 16 bytes each).  Here the warp moves 8 rows x 64 contiguous bytes per instruction instead - lane l takes
+// 16-byte piece (l & 3) of row 8 i + (l >> 2), i = 0..3 - and the two layouts meet in a per-warp buffer of
+// 32 rows x 64 bytes in which piece p of row r sits at slot p ^ ((r >> 1) & 3): both access patterns (8 rows x
+// one piece, 2 rows x 4 pieces per 128-byte wavefront) then touch every bank group once.
+// The residual of the whole block is fetched ahead of the arithmetic.
+constexpr int kEpiStageBytes = 32 * 64;  // per epilogue warp
+__device__ __forceinline__ int epi_slot(int r, int p) { return r * 64 + ((p ^ ((r >> 1) & 3)) << 4); }
+
+// 16-byte piece `piece` of the residual rows row_base + 8 i + prow, i = 0..3, columns [col0, col0 + 32)
+__device__ __forceinline__ void epi_fetch_pieces(const GemmArgs& g, int row_base, int prow, int piece, int m, int col0,
+                                                 uint4 (&dst)[4]) {
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int row = row_base + 8 * i + prow;
+    if (row < m) dst[i] = *reinterpret_cast<const uint4*>(g.resid + (size_t)row * g.ld_h + col0 + piece * 8);
+  }
+}
+
+// One 32-column chunk C of the staged epilogue (a template recursion over the chunks keeps every register array
+// statically indexed).  R[c] holds the residual pieces of chunk c, fetched by the caller.
+template <int EPI, int NC, int C>
+__device__ __forceinline__ void epi_staged_chunk(const GemmArgs& g, uint32_t taddr0, int row_base, int lane, int m, int n0,
+                                                 uint8_t* buf, uint4 (&R)[NC][4]) {
+  if constexpr (C < NC) {
+    const int prow = lane >> 2, piece = lane & 3;
+    if (EPI == EPI_HID) {
+#pragma unroll
+      for (int i = 0; i < 4; ++i) *reinterpret_cast<uint4*>(buf + epi_slot(8 * i + prow, piece)) = R[C][i];
+      __syncwarp();  // from here on a lane touches only its own row of the buffer, until the stores below
+    }
+    uint32_t r[32];
+    tc_ld32(taddr0 + (uint32_t)(C * 32), r);
+    tc_wait_ld();
+    const int col0 = n0 + C * 32;
+#pragma unroll
+    for (int e = 0; e < 32; e += 8) {
+      float x[8];
+      const float4 b0 = *reinterpret_cast<const float4*>(g.bias + col0 + e);
+      const float4 b1 = *reinterpret_cast<const float4*>(g.bias + col0 + e + 4);
+      const float bb[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
+#pragma unroll
+      for (int u = 0; u < 8; ++u) x[u] = __uint_as_float(r[e + u]) + bb[u];
+      if (EPI == EPI_HID) {
+        const uint4 rv = *reinterpret_cast<const uint4*>(buf + epi_slot(lane, e >> 3));
+        const __nv_bfloat162* rp = reinterpret_cast<const __nv_bfloat162*>(&rv);
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const float2 rf = __bfloat1622float2(rp[u]);
+          x[2 * u] = rf.x + silu(x[2 * u]);
+          x[2 * u + 1] = rf.y + silu(x[2 * u + 1]);
+        }
+      }
+      uint4 ov;
+      __nv_bfloat162* op2 = reinterpret_cast<__nv_bfloat162*>(&ov);
+#pragma unroll
+      for (int u = 0; u < 4; ++u) op2[u] = __floats2bfloat162_rn(x[2 * u], x[2 * u + 1]);
+      *reinterpret_cast<uint4*>(buf + epi_slot(lane, e >> 3)) = ov;
+    }
+    __syncwarp();
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int row = row_base + 8 * i + prow;
+      const uint4 v = *reinterpret_cast<const uint4*>(buf + epi_slot(8 * i + prow, piece));
+      if (row < m) *reinterpret_cast<uint4*>(g.out_bf16 + (size_t)row * g.ld_h + col0 + piece * 8) = v;
+    }
+    __syncwarp();
+    epi_staged_chunk<EPI, NC, C + 1>(g, taddr0, row_base, lane, m, n0, buf, R);
+  }
+}
+
+// The residual pieces of a whole 32-row x COLS-column block: they do not depend on the accumulator, so the caller
+// issues these loads BEFORE it waits for the tile's MMAs and their latency hides behind that wait.
+template <int EPI, int COLS>
+__device__ __forceinline__ void epilogue_staged_prefetch(const GemmArgs& g, int row_base, int lane, int m, int n0,
+                                                         uint4 (&R)[COLS / 32][4]) {
+  if (EPI == EPI_HID) {
+#pragma unroll
+    for (int c = 0; c < COLS / 32; ++c) epi_fetch_pieces(g, row_base, lane >> 2, lane & 3, m, n0 + c * 32, R[c]);
+  }
+}
+
+template <int EPI, int COLS>
+__device__ __forceinline__ void epilogue_tile_staged(const GemmArgs& g, uint32_t taddr0, int row_base, int lane, int m,
+                                                     int n0, uint8_t* buf, uint4 (&R)[COLS / 32][4]) {
+  static_assert(EPI != EPI_OUT, "bf16 outputs only");
+  epi_staged_chunk<EPI, COLS / 32, 0>(g, taddr0, row_base, lane, m, n0, buf, R);
 }
 
 template <int BN, int EPI>
@@ -574,7 +666,7 @@ struct PairCfg {
   static constexpr int kStageBytes = (BM + BN / 2) * BK * 2;           // per CTA: 128 rows of A, BN/2 rows of W
   static constexpr int kStages = (BN >= 256) ? 6 : (BN >= 128) ? 8 : 9;  // <= 192 KB of stages
   static constexpr int kTmemCols = 2 * BN;                             // two accumulators per CTA
-  static constexpr int kSmemBytes = kStages * kStageBytes + 1024 + 256;
+  static constexpr int kSmemBytes = kStages * kStageBytes + 1024 + 256 + kPairEpiWarps * kEpiStageBytes;
 };
 
 template <int BN, int EPI>
@@ -704,6 +796,14 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
       const int m0 = (t / tiles_n) * (2 * BM) + (int)rank * BM, n0 = (t % tiles_n) * BN;
       const int acc = it & 1;
       const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
+      constexpr int kCols = BN / (kPairEpiWarps / 4);  // this warp's share of the tile's columns
+      constexpr int kStagedCols = kCols >= 32 ? kCols : 32;
+      const int part = (warp - kEpiWarp0) >> 2;
+      // bf16 outputs of a full tile: global accesses staged through shared memory (warp-uniform choice)
+      const bool staged = EPI != EPI_OUT && kCols % 32 == 0 && n0 + BN <= g.n_out && g.ld_h % 8 == 0;
+      uint4 R[kStagedCols / 32][4];
+      if (staged)
+        epilogue_staged_prefetch<EPI == EPI_OUT ? EPI_IN : EPI, kStagedCols>(g, m0 + quarter * 32, lane, m, n0 + part * kCols, R);
       mbar_wait(accf_bar(acc), acc_phase, dead, g.err);
       tc_fence_after();
       const int row = m0 + quarter * 32 + lane;
@@ -716,10 +816,12 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
         co = g.c_out[step];
         ysrc_row = g.ysrc + (size_t)(g.row_map ? g.row_map[row] : row) * g.n_out;
       }
-      constexpr int kCols = BN / (kPairEpiWarps / 4);  // this warp's share of the tile's columns
-      const int part = (warp - kEpiWarp0) >> 2;
-      epilogue_tile<EPI, kCols>(g, tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN + part * kCols), row,
-                                row_ok, n0 + part * kCols, cs, co, ysrc_row);
+      const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN + part * kCols);
+      if (staged)
+        epilogue_tile_staged<EPI == EPI_OUT ? EPI_IN : EPI, kStagedCols>(
+            g, taddr, m0 + quarter * 32, lane, m, n0 + part * kCols, aux + 256 + (warp - kEpiWarp0) * kEpiStageBytes, R);
+      else
+        epilogue_tile<EPI, kCols, EPI == EPI_OUT>(g, taddr, row, row_ok, n0 + part * kCols, cs, co, ysrc_row);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive_cluster(map_to_cta(acce_bar(acc), 0));

@@ -160,6 +160,11 @@ struct Ctx {
   float* dbg_lr = nullptr;   // [max_chains, window]  (ASD_FLAG_DEBUG_DUMP / ASD_FLAG_DEBUG_ALL_SLOTS only)
   float* dbg_lu = nullptr;   // [max_chains, window]
   int* acc_len = nullptr;    // [max_chains]
+  float* slot_dot = nullptr; // [max_chains, window] per-slot reductions and ln u handed from the slots kernel to the verify kernel
+  float* slot_nrm = nullptr;
+  float* slot_lu = nullptr;
+  int* first_rej = nullptr;  // [max_chains] first rejected slot of the round, lowered by the slots kernel
+  int verify_horizon = -1;   // ASD_VERIFY_HORIZON at asd_create (tuning aid); -1: chosen per launch
   float* traj = nullptr;     // [max_chains, K + 1, d] (ASD_FLAG_TRAJECTORY only)
   unsigned long long* hist = nullptr;  // [window + 1] chain-rounds by accepted prefix length since the last reset
   RoundCounters* counters = nullptr;
@@ -216,6 +221,7 @@ Lane whole_batch(const Ctx* c);
 void launch_prep(Ctx* c, const Lane& L, int window);
 // v_base + (*v_off_dev) rows: where the lane's v_a rows are (v_off_dev may be null: offset 0)
 void launch_draft(Ctx* c, const Lane& L, int window, const float* v_base, const int* v_off_dev);
+int verify_horizon(const Ctx* c, int n, int window);  // slots the slots kernel reduces ahead of the verify kernel
 void launch_verify(Ctx* c, const Lane& L, int window, bool use_u, const float* G, const float* v_base,
                    const int* v_off_dev);
 // Pass-1 rows of lane L appended behind the drafted rows of the other lane: row = *row_base_dev + p gets

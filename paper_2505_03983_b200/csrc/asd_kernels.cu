@@ -20,7 +20,8 @@ __global__ void __launch_bounds__(1024) prep_kernel(const int* __restrict__ a, c
                                                     int* __restrict__ act, int* __restrict__ row_off,
                                                     int* __restrict__ step1, int* __restrict__ act1,
                                                     int* __restrict__ step1e, int* __restrict__ idx1,
-                                                    int* __restrict__ acc_len, RoundCounters* __restrict__ cnt) {
+                                                    int* __restrict__ acc_len, int* __restrict__ first_rej,
+                                                    RoundCounters* __restrict__ cnt) {
   __shared__ int s_cnt[32], s_rows[32], s_ev[32];
   __shared__ int s_base_cnt, s_base_rows, s_base_ev;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -39,6 +40,7 @@ __global__ void __launch_bounds__(1024) prep_kernel(const int* __restrict__ a, c
       rows = flag ? drafted_rows(chain_window(wnd, j, window, K, aj), aj, K, la) : 0;
       ev = flag && !(la && has_v[j]);  // v_a still has to be evaluated
       acc_len[j] = -1;
+      first_rej[j] = 0x7fffffff;  // no rejection known yet (the verify step's slots kernel lowers it)
     }
     // inclusive warp scans
     int c = flag, r = rows, e = ev;
@@ -131,7 +133,7 @@ void launch_prep(Ctx* c, const Lane& L, int window) {
   const int la = (c->lookahead && L.act1) ? 1 : 0;
   prep_kernel<<<1, 1024, 0, c->stream>>>(c->a + L.start, wnd ? wnd + L.start : nullptr, L.n, c->K, window, c->has_v, la,
                                          L.act, L.row_off, L.step1, L.act1, L.step1e, L.idx1, c->acc_len + L.start,
-                                         L.counters);
+                                         c->first_rej + L.start, L.counters);
   c->launches++;
 }
 
@@ -378,6 +380,11 @@ void launch_draft(Ctx* c, const Lane& L, int window, const float* v_base, const 
 // ---------------------------------------------------------------------------------------------
 struct VerifyArgs {
   int d, K, window, dbg_stride, nq, vec, use_u, all_slots, wps;
+  int horizon;      // slots 2 .. 1 + horizon are reduced by the slots kernel (0: none)
+  float* slot_dot;  // [n, window] per-slot <xi, delta>, |delta|^2 and ln u left by the slots kernel
+  float* slot_nrm;
+  float* slot_lu;
+  int* first_rej;   // [n] lowest rejected slot found so far this round (INT_MAX: none), lowered with atomicMin
   PhiloxKeys keys;
   uint64_t chain_base;
   RoundCounters* cnt;
@@ -406,7 +413,113 @@ struct VerifyArgs {
 
 constexpr int kVerifyMaxWarps = 8;
 
-__global__ void __launch_bounds__(256) verify_kernel(const VerifyArgs A) {
+// <xi_step, delta> and |delta|^2, delta = v_a - g, over the float4 groups tslot, tslot + team, ... of one slot
+// (a team of wps warps shares a slot); four groups per thread at a time, all their loads issued before the first use.
+// kFull: d is a multiple of 4 and every thread of the team has whole batches of four groups (no guards).
+template <bool kFull>
+__device__ __forceinline__ void slot_partial_t(const VerifyArgs& A, const float* vrow, const float* grow, uint32_t step,
+                                               uint32_t chain, int tslot, int team, float& dot, float& nrm) {
+  for (int q0 = tslot; q0 < A.nq; q0 += 4 * team) {
+    float4 vv[4], gg[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int q = q0 + u * team;
+      if (kFull) {
+        vv[u] = *reinterpret_cast<const float4*>(vrow + 4 * q);
+        gg[u] = *reinterpret_cast<const float4*>(grow + 4 * q);
+      } else if (q < A.nq) {
+        vv[u] = load4(vrow, q, A.d, A.vec);
+        gg[u] = load4(grow, q, A.d, A.vec);
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int q = q0 + u * team;
+      if (kFull || q < A.nq) {
+        const float4 xi = xi4((uint32_t)q, step, chain, A.keys);
+        float4 dl = make_float4(vv[u].x - gg[u].x, vv[u].y - gg[u].y, vv[u].z - gg[u].z, vv[u].w - gg[u].w);
+        if (!kFull && !A.vec) {  // ragged tail: dims >= d contribute nothing
+          const int b = 4 * q;
+          if (b + 1 >= A.d) dl.y = 0.f;
+          if (b + 2 >= A.d) dl.z = 0.f;
+          if (b + 3 >= A.d) dl.w = 0.f;
+        }
+        dot = fmaf(xi.x, dl.x, dot);
+        dot = fmaf(xi.y, dl.y, dot);
+        dot = fmaf(xi.z, dl.z, dot);
+        dot = fmaf(xi.w, dl.w, dot);
+        nrm = fmaf(dl.x, dl.x, nrm);
+        nrm = fmaf(dl.y, dl.y, nrm);
+        nrm = fmaf(dl.z, dl.z, nrm);
+        nrm = fmaf(dl.w, dl.w, nrm);
+      }
+    }
+  }
+}
+
+__device__ __forceinline__ void slot_partial(const VerifyArgs& A, const float* vrow, const float* grow, uint32_t step,
+                                             uint32_t chain, int tslot, int team, float& dot, float& nrm) {
+  if (A.vec && A.nq % (4 * team) == 0)  // uniform over the block
+    slot_partial_t<true>(A, vrow, grow, step, chain, tslot, team, dot, nrm);
+  else
+    slot_partial_t<false>(A, vrow, grow, step, chain, tslot, team, dot, nrm);
+}
+
+// Slots 2 .. 1 + horizon of every chain at once (the whole window for rows of some size): block (p, gy) reduces
+// the S = 8 / wps slots 2 + gy S .. of active chain p, runs their accept tests (Algorithm 3) and lowers the
+// chain's first rejected slot with atomicMin; the reductions stay in the slot arrays for the verify kernel.
+// Every block has the same work, which keeps the machine full however the accepted prefixes are spread.  Blocks
+// are dispatched in order of gy, so by the time a block of a later slot group starts, the groups before it have
+// mostly reported: a block whose chain already has a rejection below its slots leaves at once (the Verifier
+// needs nothing beyond the first rejection), which is what keeps most of the window's drifts unread.  The skip
+// only saves work: which blocks take it varies from run to run, the result does not.
+__global__ void __launch_bounds__(256, 4) verify_slots_kernel(const VerifyArgs A) {
+  __shared__ float s_part[kVerifyMaxWarps][2][kVerifyMaxWarps];  // [slot][dot | nrm][warp of team]
+  const int p = blockIdx.x;
+  if (p >= A.cnt->n_active) return;
+  const int j = A.act[p];
+  const int a = A.a[j];
+  const int w = chain_window(A.wnd, j, A.window, A.K, a);
+  const int k_end = min(w, 1 + A.horizon);
+  const int wps = A.wps, S = kVerifyMaxWarps / wps;
+  const int k_first = 2 + (int)blockIdx.y * S;
+  if (k_first > k_end) return;
+  if (!A.all_slots && *reinterpret_cast<volatile const int*>(A.first_rej + j) < k_first) return;
+  const int row0 = A.row_off[p];
+  const uint32_t chain = (uint32_t)(A.chain_base + (uint64_t)j);
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const float* vrow = (A.la && A.idx1[p] < 0) ? A.vsave + (size_t)j * A.d
+                                               : A.v + (size_t)((A.la ? A.idx1[p] : (A.v_off ? *A.v_off : 0) + p)) * A.d;
+  const int sw = warp / wps, wl = warp - sw * wps;
+  const int k = k_first + sw;
+  float dot = 0.f, nrm = 0.f;
+  if (k <= k_end)
+    slot_partial(A, vrow, A.G + (size_t)(row0 + k - 2) * A.d, (uint32_t)(a + k), chain, wl * 32 + lane, wps * 32, dot, nrm);
+  dot = warp_sum(dot);
+  nrm = warp_sum(nrm);
+  if (lane == 0) {
+    s_part[sw][0][wl] = dot;
+    s_part[sw][1][wl] = nrm;
+  }
+  __syncthreads();
+  if (tid < S && k_first + tid <= k_end) {
+    float d2 = 0.f, n2 = 0.f;
+    for (int x = 0; x < wps; ++x) {
+      d2 += s_part[tid][0][x];
+      n2 += s_part[tid][1][x];
+    }
+    const int kk = k_first + tid, i = a + kk - 1;
+    const size_t o = (size_t)j * A.dbg_stride + kk - 1;
+    const float lu = A.use_u ? ln_u((uint32_t)(a + kk), chain, A.keys) : 0.f;
+    A.slot_dot[o] = d2;
+    A.slot_nrm[o] = n2;
+    A.slot_lu[o] = lu;
+    const float lr = ln_ratio_of(A.tab.c1[i], A.tab.c2[i], d2, n2);
+    if (!((lu <= fminf(0.f, lr)) || (n2 == 0.f))) atomicMin(A.first_rej + j, kk);
+  }
+}
+
+__global__ void __launch_bounds__(256, 3) verify_kernel(const VerifyArgs A) {
   __shared__ float s_part[2][kVerifyMaxWarps][2][kVerifyMaxWarps];  // [group parity][slot][dot | nrm][warp of team]
   __shared__ float s_lu[2][kVerifyMaxWarps];                        // [group parity][slot] ln u
   const int p = blockIdx.x;
@@ -428,58 +541,43 @@ __global__ void __launch_bounds__(256) verify_kernel(const VerifyArgs A) {
       A.dbg_lu[(size_t)j * A.dbg_stride + k - 1] = A.use_u ? ln_u((uint32_t)(a + k), chain, A.keys) : 0.f;
       A.dbg_lr[(size_t)j * A.dbg_stride + k - 1] = k == 1 ? 0.f : nan;
     }
+    __syncthreads();  // the values written below replace these
   }
 
-  // Slots are taken in groups of S = nwarps / wps; a team of wps warps reduces one slot.
+  int n = w;                  // accepted prefix length; w = no rejection seen
+  float rej_dot = 0.f, rej_nrm = 1.f;
+  // slots 2 .. k_par went through the slots kernel: every slot up to the chain's first rejection was reduced and
+  // tested there (and every slot of the window in the all-slots mode)
+  const int k_par = min(w, 1 + A.horizon);
+  if (k_par >= 2) {
+    const int first = A.first_rej[j];
+    if (first <= k_par) {
+      n = first - 1;
+      rej_dot = A.slot_dot[(size_t)j * A.dbg_stride + first - 1];
+      rej_nrm = A.slot_nrm[(size_t)j * A.dbg_stride + first - 1];
+    }
+    if (A.dbg_lr) {
+      const int k_have = A.all_slots ? k_par : min(first, k_par);
+      for (int k = 2 + tid; k <= k_have; k += blockDim.x) {
+        const size_t o = (size_t)j * A.dbg_stride + k - 1;
+        const int i = a + k - 1;
+        A.dbg_lr[o] = ln_ratio_of(A.tab.c1[i], A.tab.c2[i], A.slot_dot[o], A.slot_nrm[o]);
+      }
+    }
+  }
+
+  // Beyond them the slots are taken in groups of S = nwarps / wps (a team of wps warps reduces one slot), in order,
+  // and the walk stops after the group that holds the first rejection.
   const int wps = A.wps, S = nwarps / wps;
   const int sw = warp / wps, wl = warp - sw * wps;
   const int tslot = wl * 32 + lane, team = wps * 32;
-  int n = w;                  // accepted prefix length; w = no rejection seen
-  float rej_dot = 0.f, rej_nrm = 1.f;
-  int par = 0, rows_read = 0;
-  for (int k0 = 2; k0 <= w; k0 += S, par ^= 1) {
+  int par = 0;
+  for (int k0 = max(2, k_par + 1); k0 <= w && n == w; k0 += S, par ^= 1) {
     const int k = k0 + sw;
-    rows_read = min(k0 + S - 1, w) - 1;
     // ln u of the group's slots (one Philox call each), by the first S threads
     if (tid < S && k0 + tid <= w) s_lu[par][tid] = A.use_u ? ln_u((uint32_t)(a + k0 + tid), chain, A.keys) : 0.f;
     float dot = 0.f, nrm = 0.f;
-    if (k <= w) {
-      const float* grow = A.G + (size_t)(row0 + k - 2) * A.d;
-      // four float4 groups per thread at a time: all their loads are issued before the first use
-      for (int q0 = tslot; q0 < A.nq; q0 += 4 * team) {
-        float4 vv[4], gg[4];
-#pragma unroll
-        for (int u = 0; u < 4; ++u) {
-          const int q = q0 + u * team;
-          if (q < A.nq) {
-            vv[u] = load4(vrow, q, A.d, A.vec);
-            gg[u] = load4(grow, q, A.d, A.vec);
-          }
-        }
-#pragma unroll
-        for (int u = 0; u < 4; ++u) {
-          const int q = q0 + u * team;
-          if (q < A.nq) {
-            const float4 xi = xi4((uint32_t)q, (uint32_t)(a + k), chain, A.keys);
-            float4 dl = make_float4(vv[u].x - gg[u].x, vv[u].y - gg[u].y, vv[u].z - gg[u].z, vv[u].w - gg[u].w);
-            if (!A.vec) {  // ragged tail: dims >= d contribute nothing
-              const int b = 4 * q;
-              if (b + 1 >= A.d) dl.y = 0.f;
-              if (b + 2 >= A.d) dl.z = 0.f;
-              if (b + 3 >= A.d) dl.w = 0.f;
-            }
-            dot = fmaf(xi.x, dl.x, dot);
-            dot = fmaf(xi.y, dl.y, dot);
-            dot = fmaf(xi.z, dl.z, dot);
-            dot = fmaf(xi.w, dl.w, dot);
-            nrm = fmaf(dl.x, dl.x, nrm);
-            nrm = fmaf(dl.y, dl.y, nrm);
-            nrm = fmaf(dl.z, dl.z, nrm);
-            nrm = fmaf(dl.w, dl.w, nrm);
-          }
-        }
-      }
-    }
+    if (k <= w) slot_partial(A, vrow, A.G + (size_t)(row0 + k - 2) * A.d, (uint32_t)(a + k), chain, tslot, team, dot, nrm);
     dot = warp_sum(dot);
     nrm = warp_sum(nrm);
     if (lane == 0) {
@@ -488,7 +586,6 @@ __global__ void __launch_bounds__(256) verify_kernel(const VerifyArgs A) {
     }
     __syncthreads();
     // every thread walks the group's slots in order and so reaches the same decision
-    bool stop = false;
     for (int s2 = 0; s2 < S && k0 + s2 <= w; ++s2) {
       float d2 = 0.f, n2 = 0.f;
       for (int x = 0; x < wps; ++x) {
@@ -503,14 +600,15 @@ __global__ void __launch_bounds__(256) verify_kernel(const VerifyArgs A) {
         n = kk - 1;
         rej_dot = d2;
         rej_nrm = n2;
-        if (!A.all_slots) {
-          stop = true;
-          break;
-        }
+        break;
       }
     }
-    if (stop) break;
   }
+
+  // the drift rows an in-order walk in groups of S slots reads: up to the end of the group with the first rejection
+  // (what the slots kernel really read depends on which of its blocks could leave early; never less than this)
+  int rows_read = 0;
+  if (w >= 2) rows_read = (n == w || A.all_slots) ? w - 1 : min(2 + ((n + 1 - 2) / S) * S + S - 1, w) - 1;
 
   float* yrow = A.y + (size_t)j * A.d;
   if (n < w) {
@@ -591,6 +689,18 @@ __global__ void __launch_bounds__(256) verify_kernel(const VerifyArgs A) {
   }
 }
 
+// How many slots after slot 1 go through the slots kernel (all chains and slot groups side by side): the whole
+// window, except for rows of a few hundred floats, where the extra launch would cost more than it saves and the
+// verify kernel walks the slots itself.  ASD_VERIFY_HORIZON (read at asd_create) overrides it for experiments.
+int verify_horizon(const Ctx* c, int n, int window) {
+  (void)n;
+  if (window < 2) return 0;
+  if (c->debug_all_slots) return window - 1;  // that mode tests every slot, which only the slots kernel does
+  if (c->verify_horizon >= 0) return std::min(c->verify_horizon, window - 1);
+  if (c->d < 256) return 0;
+  return window - 1;
+}
+
 void launch_verify(Ctx* c, const Lane& L, int window, bool use_u, const float* G, const float* v_base,
                    const int* v_off_dev) {
   if (L.n == 0) return;
@@ -630,6 +740,16 @@ void launch_verify(Ctx* c, const Lane& L, int window, bool use_u, const float* G
   A.hist = c->hist;
   // eight warps per chain; a slot is reduced by two warps when a row has >= 512 float4 groups, else by one
   A.wps = A.nq >= 512 ? 2 : 1;
+  A.horizon = verify_horizon(c, L.n, window);
+  A.slot_dot = c->slot_dot + (size_t)L.start * c->window;
+  A.slot_nrm = c->slot_nrm + (size_t)L.start * c->window;
+  A.slot_lu = c->slot_lu + (size_t)L.start * c->window;
+  A.first_rej = c->first_rej + L.start;
+  if (A.horizon > 0) {
+    const int S = kVerifyMaxWarps / A.wps;
+    verify_slots_kernel<<<dim3(L.n, (A.horizon + S - 1) / S), 256, 0, c->stream>>>(A);
+    c->launches++;
+  }
   verify_kernel<<<L.n, 256, 0, c->stream>>>(A);
   c->launches++;
 }
