@@ -495,6 +495,11 @@ def run_ours(args):
             else:
                 w4 = workloads.make(name)
             cfgs[name] = compact_config(torch, AsdSampler, w4, peaks)
+        # the cfg-1 problem with a small network fitted to its closed-form posterior mean (stored weights): rounds per
+        # sample on a true posterior mean represented by the bf16 network, next to the closed form's (cfg1_gmm2d)
+        wt = workloads.make("cfg1_trained", chains=256)
+        cfgs["cfg1_trained_mlp_256_chains"] = compact_config(torch, AsdSampler, wt, peaks)
+        cfgs["cfg1_gmm2d_256_chains"] = compact_config(torch, AsdSampler, workloads.make("cfg1_gmm2d", chains=256), peaks)
         line["configs"] = cfgs
     print(json.dumps(line))
     if dist is not None:

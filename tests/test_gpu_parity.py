@@ -869,3 +869,26 @@ def test_lockstep_resident_kernel_rounds(name, chains, rounds, kw, adaptive, mon
         st = s.round()
         assert st.rows_pass1 == st.n_active_before
     assert worst["decided"] > 0
+
+
+def test_trained_network_lockstep_and_rounds():
+    """The cfg-1 problem with the small network that was fitted to its posterior mean (stored weights): lock-step
+    parity like any network, and over whole runs about as many rounds per sample as with the closed form itself
+    (the acceptance behaviour of a true posterior mean, not of a random network)."""
+    wl = workloads.make("cfg1_trained", chains=64)
+    with _sampler(wl) as s:
+        worst = lockstep(s, wl, 64, 12, chain_base=50, log=_log)
+        s.reset(64, 50)
+        y, r, st = s.sample()
+    base = workloads.make("cfg1_gmm2d", chains=64)
+    with _sampler(base, dump=False) as s0:
+        s0.reset(64, 50)
+        y0, r0, st0 = s0.sample()
+    _log(f"rounds per sample: fitted network {st.rounds_mean:.2f}, closed form {st0.rounds_mean:.2f}")
+    assert worst["decided"] > 0 and torch.isfinite(y).all()
+    assert abs(st.rounds_mean - st0.rounds_mean) < 0.25 * st0.rounds_mean
+    # most chains end in the same mixture component as with the closed form (same noise streams)
+    T = base.t[-1]
+    c = torch.as_tensor(base.means, device="cuda")
+    lab = lambda yy: torch.argmin(((yy[:, None, :] / T - c[None]) ** 2).sum(-1), dim=1)
+    assert (lab(y) == lab(y0)).float().mean() > 0.8

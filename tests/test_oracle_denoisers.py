@@ -168,3 +168,26 @@ def test_resmlp_batch_rows_match_single_calls_mixed_steps(name):
         assert not np.allclose(g.batch([5] * len(steps), Y, chain), got)
         if wl.d_cond:
             assert not np.allclose(g.batch(steps, Y, (chain + 1) % wl.chains), got)
+
+
+def test_stored_trained_network_approximates_the_mixture_posterior_mean():
+    """tests/golden/cfg1_trained_mlp.npz (written by tests/golden/make_cfg1_trained_mlp.py) is a network fitted
+    to Eq. 4's posterior mean of the cfg-1 mixture: on fresh points of the localization process its drift is
+    close to the closed form, far closer than the skip term alone."""
+    wl = workloads.make("cfg1_trained")
+    base = workloads.make("cfg1_gmm2d")
+    net, exact = den.from_workload(wl), den.from_workload(base)
+    rng = np.random.default_rng(123)
+    err, err_skip, ref = [], [], []
+    for _ in range(400):
+        i = int(rng.integers(0, wl.K))
+        xs = base.means[rng.integers(0, 8)] + base.sigma * rng.standard_normal(2)
+        y = base.t[i] * xs + math.sqrt(base.t[i]) * rng.standard_normal(2)
+        m = exact(i, y)
+        err.append(np.sum((net(i, y) - m) ** 2))
+        err_skip.append(np.sum((float(wl.c_skip[i]) * y - m) ** 2))
+        ref.append(np.sum(m ** 2))
+    rel = math.sqrt(np.sum(err) / np.sum(ref))
+    rel_skip = math.sqrt(np.sum(err_skip) / np.sum(ref))
+    print(f"trained network: rms error / rms posterior mean = {rel:.3f} (skip term alone {rel_skip:.3f})")
+    assert rel < 0.1 and rel < 0.2 * rel_skip

@@ -15,6 +15,7 @@ Workloads (synthetic stand-ins, no dataset or trained weight is used):
   cfg4_image     d=3x32x32=3072, 6-layer residual MLP width 4096, K=1000, window 32, 32 chains
   sweep_b{B}_w{W}  cfg4 denoiser, B chains x window W, K=1000
   mlp_tiny / mlp_ragged   small residual-MLP cases for parity tests (several tiles + ragged tails)
+  cfg1_trained   the cfg-1 problem with a small residual MLP fitted to its posterior mean (stored weights)
 
 All time grids are the uniform stochastic-localization grid t_i = i*T/K with
 T = 100 ("linear schedule"), the equal-increment case of the exchangeability
@@ -162,6 +163,18 @@ def make(name: str, *, chains: Optional[int] = None, K: Optional[int] = None,
     if m:
         return _mlp(name, 3072, 0, 256, 4096, ov(n_layers, 6), ov(K, 1000), ov(window, int(m.group(2))),
                     ov(chains, int(m.group(1))), s)
+    if name == "cfg1_trained":
+        # the cfg-1 problem with a small network FITTED to the mixture's closed-form posterior mean in place of the
+        # closed form (weights and per-step tables as stored by tests/golden/make_cfg1_trained_mlp.py)
+        import os
+        z = np.load(os.path.join(os.path.dirname(os.path.abspath(__file__)), "tests", "golden", "cfg1_trained_mlp.npz"))
+        Kc = ov(K, 100)
+        assert Kc == len(z["c_in"]), "the stored per-step tables are for K = 100"
+        return Workload(name=name, kind="mlp", d=2, K=Kc, window=ov(window, 8), chains=ov(chains, 16), seed=s,
+                        t=uniform_grid(Kc), d_cond=0, d_temb=int(z["d_temb"]), width=z["W_in"].shape[0],
+                        n_layers=z["W_hid"].shape[0], W_in=z["W_in"], W_hid=z["W_hid"], W_out=z["W_out"],
+                        b_in=z["b_in"], b_hid=z["b_hid"], b_out=z["b_out"], c_in=z["c_in"], c_skip=z["c_skip"],
+                        c_out=z["c_out"], cond=np.zeros((ov(chains, 16), 0), np.float32))
     if name == "mlp_tiny":
         return _mlp(name, 24, 8, 32, 128, 2, ov(K, 40), ov(window, 6), ov(chains, 5), s, bias_std=0.05)
     if name == "mlp_ragged":
