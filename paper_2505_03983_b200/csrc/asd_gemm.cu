@@ -922,6 +922,15 @@ gemm_skinny_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
+  // What the fused tail reads from global memory does not depend on this kernel's own product: the epilogue warps
+  // fetch it (row count, bias, and the residual / state / per-row scalars of their first group of rows) while the
+  // weights are still streaming, instead of after the cluster's partials are in place.
+  constexpr int kSkR = 8;  // rows per group of the reduction below
+  int m_pre = 0;
+  float bias_pre = 0.f, opnd_pre[kSkR], cs_pre[kSkR], co_pre[kSkR];
+#pragma unroll
+  for (int u = 0; u < kSkR; ++u) opnd_pre[u] = cs_pre[u] = co_pre[u] = 0.f;
+
   if (warp == 0) {
     // ---------------- TMA producer ----------------
     if (lane == 0) {
@@ -983,6 +992,28 @@ gemm_skinny_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
     // ---- park this rank's partial D^T[feature, row] in shared memory as part[row][feature] ----
     const int quarter = warp & 3;
     const int feat = quarter * 32 + lane;  // tensor-memory lane = feature within the tile
+    {
+      grid_dependency_wait();  // the row count, the residual and the state come from earlier kernels
+      m_pre = max(0, min(min(*g.m_dev, g.m_cap) - row0, m_pad));
+      const int n = n0 + feat;
+      if (n < g.n_out && m_pre > 0) {
+        bias_pre = g.bias[n];
+        const int kRowStep = kSplit * (((int)(blockDim.x >> 5) - kEpiWarp0) >> 2);
+        const int lr_first = (int)rank + ((warp - kEpiWarp0) >> 2) * kSplit;
+#pragma unroll
+        for (int u = 0; u < kSkR; ++u) {
+          const int row = row0 + min(lr_first + u * kRowStep, m_pre - 1);
+          if (EPI == EPI_OUT) {
+            const int step = g.row_step[row];
+            cs_pre[u] = g.c_skip[step];
+            co_pre[u] = g.c_out[step];
+            opnd_pre[u] = g.ysrc[(size_t)(g.row_map ? g.row_map[row] : row) * g.n_out + n];
+          } else if (EPI == EPI_HID) {
+            opnd_pre[u] = __bfloat162float(g.resid[(size_t)row * g.ld_h + n]);
+          }
+        }
+      }
+    }
     mbar_wait(accf_bar, 0u, dead, g.err);
     tc_fence_after();
     float* part = reinterpret_cast<float*>(tiles_ptr);  // the stage buffers are idle now: [m_pad][128] fp32
@@ -1011,21 +1042,22 @@ gemm_skinny_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
     const int quarter = warp & 3;
     const int feat = quarter * 32 + lane;
     const int n = n0 + feat;
-    grid_dependency_wait();  // the row count, the residual and the state come from earlier kernels
-    const int m = max(0, min(min(*g.m_dev, g.m_cap) - row0, m_pad));
+    const int m = m_pre;
     if (n < g.n_out) {
       uint32_t part_of[kSplit];  // the partial buffer sits at the same offset in every CTA of the cluster
 #pragma unroll
       for (int q = 0; q < kSplit; ++q) part_of[q] = map_to_cta(tiles, (uint32_t)q);
-      const float bias = g.bias[n];
+      const float bias = bias_pre;
       // rows rank, rank + kSplit, ... of the block, eight at a time: all their loads (partials over
       // distributed shared memory, residual / state and per-row scalars from global memory) are issued
       // before the first store, so one memory latency is paid per group instead of per row
-      constexpr int R = 8;
+      constexpr int R = kSkR;
       const int kRowStep = kSplit * (((int)(blockDim.x >> 5) - kEpiWarp0) >> 2);  // this warp's rows: every kRowStep-th
       const int half = (warp - kEpiWarp0) >> 2;
-      for (int lr0 = (int)rank + half * kSplit; lr0 < m; lr0 += R * kRowStep) {
+      const int lr_first = (int)rank + half * kSplit;
+      for (int lr0 = lr_first; lr0 < m; lr0 += R * kRowStep) {
         float acc[R], opnd[R], cs[R], co[R];
+        const bool first = lr0 == lr_first;  // this group's operands were fetched ahead
 #pragma unroll
         for (int u = 0; u < R; ++u) {
           const int lr = min(lr0 + u * kRowStep, m - 1);  // clamped rows are loaded but not stored
@@ -1034,7 +1066,11 @@ gemm_skinny_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
 #pragma unroll
           for (int q = 0; q < kSplit; ++q) a += ld_cluster_f32(part_of[q] + (uint32_t)((lr * BM + feat) * 4));
           acc[u] = a;
-          if (EPI == EPI_OUT) {
+          if (first) {
+            opnd[u] = opnd_pre[u];
+            cs[u] = cs_pre[u];
+            co[u] = co_pre[u];
+          } else if (EPI == EPI_OUT) {
             const int step = g.row_step[row];
             cs[u] = g.c_skip[step];
             co[u] = g.c_out[step];

@@ -873,11 +873,17 @@ def test_lockstep_resident_kernel_rounds(name, chains, rounds, kw, adaptive, mon
 
 def test_trained_network_lockstep_and_rounds():
     """The cfg-1 problem with the small network that was fitted to its posterior mean (stored weights): lock-step
-    parity like any network, and over whole runs about as many rounds per sample as with the closed form itself
-    (the acceptance behaviour of a true posterior mean, not of a random network)."""
+    parity, and over whole runs about as many rounds per sample as with the closed form itself (the acceptance
+    behaviour of a true posterior mean, not of a random network).  This network carries the whole drift (c_out of
+    order 1, trained weights of order 1), so it is as sensitive as a network can be to the bf16 rounding of its
+    two inputs: the library's fp32 drafted point and the oracle's fp64 one differ by 1e-7 relative, which now and
+    then rounds c_in y to the neighbouring bf16 value and moves the network branch by up to a few per cent
+    (tests/test_bf16_cascade_cpu.py shows the mechanism on the CPU).  ln ratio is therefore compared at the
+    bf16-resolution bound of tests/_parity.py and the share of exempt decisions is bounded."""
     wl = workloads.make("cfg1_trained", chains=64)
     with _sampler(wl) as s:
-        worst = lockstep(s, wl, 64, 12, chain_base=50, log=_log)
+        worst = lockstep(s, wl, 64, 12, chain_base=50, log=_log, cascade=True)
+        assert worst["exempt"] <= 0.25 * (worst["exempt"] + worst["decided"])
         s.reset(64, 50)
         y, r, st = s.sample()
     base = workloads.make("cfg1_gmm2d", chains=64)
