@@ -544,6 +544,8 @@ asd_status asd_create(const asd_config* cfg, void* cuda_stream, asd_ctx** out) {
     c->use_graphs = !(e && e[0] == '0');
     const char* gm = getenv("ASD_GEMM_MODE");  // tuning aid: pins the GEMM kernel family
     c->gemm_mode = !gm ? 0 : (!strcmp(gm, "cta") ? 1 : (!strcmp(gm, "pair") ? 2 : 0));
+    const char* fm = getenv("ASD_MLP_FUSED");  // "1": the whole network as one launch (measured slower; see asd_gemm.cu)
+    c->fused_mode = (fm && fm[0] == '1') ? 1 : 0;
     const char* sg = getenv("ASD_STAGGER");
     c->stagger = sg && sg[0] == '1';
     const char* vh = getenv("ASD_VERIFY_HORIZON");  // tuning aid: slots verified for all chains at once (default: per launch)

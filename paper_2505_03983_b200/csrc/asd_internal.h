@@ -183,6 +183,8 @@ struct Ctx {
   std::map<std::tuple<const void*, int, int, int>, CUtensorMap> tmaps;
   std::map<const void*, int> func_smem;  // kernel -> dynamic shared memory opted in on this context's device
   int gemm_mode = 0;                     // ASD_GEMM_MODE at asd_create: 0 planner, 1 "cta", 2 "pair"
+  int fused_ready = 0, fused_clusters = 0;  // one-launch network: 0 not yet checked, 1 usable, -1 not; clusters that fit the device at once
+  int fused_mode = -1;                   // ASD_MLP_FUSED=1 at asd_create: the whole network in one launch (off otherwise)
   bool stagger = false;                  // ASD_STAGGER=1 at asd_create
   int resident_mode = 1;                 // ASD_RESIDENT at asd_create: 0 never, 1 asd_sample / asd_sequential_ddpm, 2 asd_round too
   // One speculation round captured as a CUDA graph per (window, use_u, bound on active chains); replayed

@@ -898,3 +898,29 @@ def test_trained_network_lockstep_and_rounds():
     c = torch.as_tensor(base.means, device="cuda")
     lab = lambda yy: torch.argmin(((yy[:, None, :] / T - c[None]) ** 2).sum(-1), dim=1)
     assert (lab(y) == lab(y0)).float().mean() > 0.8
+
+
+@pytest.mark.parametrize("name,chains,rounds", [("mlp_ragged", 37, 8), ("cfg3_policy", 64, 4), ("mlp_odd", 7, 6)])
+def test_one_launch_network_kernel(name, chains, rounds, monkeypatch):
+    """ASD_MLP_FUSED=1: the whole network in one launch (a cluster of CTAs per 128 rows, the layers chained by
+    cluster barriers).  Off by default because it measured slower; kept correct: the drift against the oracle on
+    row counts with ragged row blocks, and lock-step rounds."""
+    monkeypatch.setenv("ASD_MLP_FUSED", "1")
+    wl = workloads.make(name, chains=chains)
+    cond = wl.cond if wl.d_cond else None
+    rng = np.random.default_rng(2)
+    g = oden.from_workload(wl)
+    with _sampler(wl) as s:
+        s.reset(chains, 0, cond=cond)
+        cap = chains * (wl.window - 1)
+        for n_rows in (1, min(130, cap), cap):
+            steps = rng.integers(0, wl.K, n_rows).astype(np.int32)
+            y = (wl.t[steps][:, None] * rng.standard_normal((n_rows, wl.d)) +
+                 np.sqrt(wl.t[steps])[:, None] * rng.standard_normal((n_rows, wl.d))).astype(np.float32)
+            slots = rng.integers(0, chains, n_rows).astype(np.int32)
+            out = s.denoise(steps, y, slots).cpu().numpy()
+            for r in np.unique(np.concatenate([[0, n_rows - 1, n_rows // 2], rng.integers(0, n_rows, 20)])):
+                ref = g(int(steps[r]), y[r].astype(np.float64), int(slots[r]))
+                assert np.max(np.abs(out[r] - ref)) / max(1.0, np.max(np.abs(ref))) < 2e-3
+        worst = lockstep(s, wl, chains, rounds, chain_base=60, cond=cond, log=_log)
+    assert worst["decided"] > 0
