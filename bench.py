@@ -33,7 +33,7 @@ DEFAULT_WORKLOAD = "sweep_b512_w64"   # cfg-4 denoiser, 512 chains x window 64, 
 # dram__bytes_read.sum + dram__bytes_write.sum of one pass-2 hidden-layer launch of gemm_pair_kernel<256, EPI_HID>
 # at full row count, from one ncu capture of that kernel; set an entry to None when the kernel changes, until the
 # counters are taken again
-NCU_TRAFFIC_BYTES_PER_LAUNCH = {"sweep_b512_w64": 391_901_184 + 244_783_872}
+NCU_TRAFFIC_BYTES_PER_LAUNCH = {"sweep_b512_w64": 390_400_000 + 246_830_000}
 METRIC = "samples_per_sec"
 UNIT = "samples/s"
 
@@ -500,6 +500,10 @@ def run_ours(args):
         wt = workloads.make("cfg1_trained", chains=256)
         cfgs["cfg1_trained_mlp_256_chains"] = compact_config(torch, AsdSampler, wt, peaks)
         cfgs["cfg1_gmm2d_256_chains"] = compact_config(torch, AsdSampler, workloads.make("cfg1_gmm2d", chains=256), peaks)
+        # theta = infinity (window = K: every round drafts to the end of the grid), the paper's upper limit of the
+        # algorithmic speed-up
+        cfgs["cfg1_gmm2d_theta_inf"] = compact_config(torch, AsdSampler, workloads.make("cfg1_gmm2d", window=100), peaks)
+        cfgs["cfg2_gauss64_theta_inf"] = compact_config(torch, AsdSampler, workloads.make("cfg2_gauss64", window=1000, chains=64), peaks)
         line["configs"] = cfgs
     print(json.dumps(line))
     if dist is not None:
@@ -520,12 +524,15 @@ def main():
     ap.add_argument("--profile-rounds", type=int, default=0,
                     help="profiling aid: reset, run this many speculation rounds, print nothing timed and exit "
                          "(a short, bounded launch sequence for ncu captures)")
+    ap.add_argument("--all-slots", action="store_true",
+                    help="with --profile-rounds: create the sampler with ASD_FLAG_DEBUG_ALL_SLOTS (every window slot verified)")
     args = ap.parse_args()
     if args.profile_rounds > 0:
         import torch
         from paper_2505_03983_b200 import AsdSampler
+        from paper_2505_03983_b200.binding import FLAG_DEBUG_ALL_SLOTS
         wl = workloads.make(args.workload)
-        with AsdSampler(wl) as s:
+        with AsdSampler(wl, flags=FLAG_DEBUG_ALL_SLOTS if args.all_slots else 0) as s:
             cond = torch.as_tensor(wl.cond, device="cuda") if wl.kind == "mlp" and wl.d_cond else None
             s.reset(wl.chains, 0, cond=cond)
             for _ in range(args.profile_rounds):

@@ -10,7 +10,7 @@ v_a = g(t_a, y_a), proposal means m^_{i+1} = y^_i + eta_i v_a, proposal samples
 y^_{i+1} = m^_{i+1} + sigma_{i+1} xi_{i+1}, target means
 m_{i+1} = y^_i + eta_i g(t_i, y^_i).
 
-Readings of the paper taken here (each also listed in the design notes):
+Readings of the paper taken here:
  * step size eta_i = t_{i+1} - t_i (Eq. 3; the definition under Eq. 7 has a typo);
  * the Gaussians of Eq. 8 / Eq. 9 have covariance sigma_{i+1}^2 I as in Algorithm 1;
    in the stochastic-localization chain sigma_{i+1}^2 = eta_i (increments given x*

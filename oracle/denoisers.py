@@ -26,7 +26,8 @@ ResMlpDenoiser        the synthetic network of the bf16 workloads.  The paper do
 Pins (tests/test_oracle_denoisers.py): both closed forms against numerical
 integration of the defining conditional expectation (d = 1 and 2), the GMM form
 at t = 0 (prior mean) and for one component (Gaussian form), the network against
-a plain triple loop, and bf16 rounding against torch's cast.
+a plain triple loop, its batched form (several rows, a different step per row)
+against the single-point form, and bf16 rounding against torch's cast.
 """
 from __future__ import annotations
 

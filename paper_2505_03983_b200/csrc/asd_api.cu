@@ -37,6 +37,9 @@ template <typename T>
 asd_status dev_alloc(Ctx* c, T** out, size_t count, bool zero = true) {
   void* p = nullptr;
   const size_t bytes = std::max<size_t>(count, 1) * sizeof(T);
+  // host-side failure injection for the tests of the error path (ASD_FAIL_ALLOC_AFTER=n at asd_create)
+  if (c->fail_alloc_after >= 0 && (int)c->dev_allocs.size() >= c->fail_alloc_after)
+    return fail(c, ASD_ERR_OOM, "cudaMalloc: injected allocation failure");
   cudaError_t e = cudaMalloc(&p, bytes);
   if (e != cudaSuccess) return fail(c, ASD_ERR_OOM, std::string("cudaMalloc: ") + cudaGetErrorString(e));
   c->dev_allocs.push_back(p);
@@ -548,6 +551,8 @@ asd_status asd_create(const asd_config* cfg, void* cuda_stream, asd_ctx** out) {
     c->fused_mode = (fm && fm[0] == '1') ? 1 : 0;
     const char* sg = getenv("ASD_STAGGER");
     c->stagger = sg && sg[0] == '1';
+    const char* fa = getenv("ASD_FAIL_ALLOC_AFTER");  // test hook: the n-th device allocation of this context fails
+    c->fail_alloc_after = fa ? atoi(fa) : -1;
     const char* vh = getenv("ASD_VERIFY_HORIZON");  // tuning aid: slots verified for all chains at once (default: per launch)
     c->verify_horizon = vh ? atoi(vh) : -1;
     const char* rm = getenv("ASD_RESIDENT");  // tuning aid: "0" keeps the closed-form drifts on the per-phase kernels

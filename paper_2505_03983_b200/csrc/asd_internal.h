@@ -164,6 +164,7 @@ struct Ctx {
   float* slot_nrm = nullptr;
   float* slot_lu = nullptr;
   int* first_rej = nullptr;  // [max_chains] first rejected slot of the round, lowered by the slots kernel
+  int fail_alloc_after = -1; // ASD_FAIL_ALLOC_AFTER at asd_create (test hook): device allocations that succeed before one fails
   int verify_horizon = -1;   // ASD_VERIFY_HORIZON at asd_create (tuning aid); -1: chosen per launch
   float* traj = nullptr;     // [max_chains, K + 1, d] (ASD_FLAG_TRAJECTORY only)
   unsigned long long* hist = nullptr;  // [window + 1] chain-rounds by accepted prefix length since the last reset

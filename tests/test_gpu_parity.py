@@ -924,3 +924,27 @@ def test_one_launch_network_kernel(name, chains, rounds, monkeypatch):
                 assert np.max(np.abs(out[r] - ref)) / max(1.0, np.max(np.abs(ref))) < 2e-3
         worst = lockstep(s, wl, chains, rounds, chain_base=60, cond=cond, log=_log)
     assert worst["decided"] > 0
+
+
+@pytest.mark.parametrize("name", ["cfg1_gmm2d", "mlp_tiny"])
+def test_allocation_failure_is_reported_and_leaves_nothing_behind(name, monkeypatch):
+    """Failure path of asd_create, injected on the host: the n-th device allocation of the context fails.  The call
+    returns ASD_ERR_OOM with a message, frees what it had allocated, and the next context works as usual."""
+    from paper_2505_03983_b200 import AsdError
+    wl = workloads.make(name)
+    cond = wl.cond if wl.kind == "mlp" and wl.d_cond else None
+    with _sampler(wl, dump=False) as s:
+        s.reset(wl.chains, 0, cond=cond)
+        y_ref, r_ref, _ = s.sample()
+    free0 = torch.cuda.mem_get_info()[0]
+    for n in (0, 1, 4, 9, 17, 24):
+        monkeypatch.setenv("ASD_FAIL_ALLOC_AFTER", str(n))
+        with pytest.raises(AsdError) as e:
+            _sampler(wl, dump=False)
+        assert e.value.status == 3 and "allocation" in str(e.value)
+    monkeypatch.delenv("ASD_FAIL_ALLOC_AFTER")
+    assert torch.cuda.mem_get_info()[0] >= free0 - (8 << 20)          # nothing of the failed contexts is left
+    with _sampler(wl, dump=False) as s:
+        s.reset(wl.chains, 0, cond=cond)
+        y, r, _ = s.sample()
+    assert torch.equal(y, y_ref) and torch.equal(r, r_ref)
