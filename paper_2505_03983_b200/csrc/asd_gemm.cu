@@ -510,6 +510,62 @@ __device__ __forceinline__ void epilogue_tile_staged(const GemmArgs& g, uint32_t
   epi_staged_chunk<EPI, COLS / 32, 0>(g, taddr0, row_base, lane, m, n0, buf, R);
 }
 
+// The same staging for the output projection (fp32 in, fp32 out): a 32-column chunk is taken as two halves of 16
+// columns = 64 bytes per row, the geometry of the bf16 path.  Per half the warp fetches the state rows y (through the
+// optional row map) 8 rows x 64 contiguous bytes per instruction, hands them to the lanes that own the rows, and
+// writes g = c_skip y + c_out (acc + b) the same way.  The state pieces of the next half are in flight during the
+// arithmetic of the current one.
+template <int COLS>
+__device__ __forceinline__ void epilogue_tile_staged_out(const GemmArgs& g, uint32_t taddr0, int row_base, int lane, int m,
+                                                         int n0, uint8_t* buf, float cs, float co) {
+  constexpr int NH = COLS / 16;  // halves
+  const int prow = lane >> 2, piece = lane & 3;
+  const float* yrow[4];  // state rows of the tile rows 8 i + prow (null: beyond the valid rows)
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int row = row_base + 8 * i + prow;
+    yrow[i] = row < m ? g.ysrc + (size_t)(g.row_map ? g.row_map[row] : row) * g.n_out : nullptr;
+  }
+  uint4 Y[2][4];
+  auto fetch = [&](int h, uint4 (&dst)[4]) {
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+      if (yrow[i]) dst[i] = *reinterpret_cast<const uint4*>(yrow[i] + n0 + h * 16 + piece * 4);
+  };
+  fetch(0, Y[0]);
+  uint32_t r[32];
+#pragma unroll
+  for (int h = 0; h < NH; ++h) {
+    if ((h & 1) == 0) tc_ld32(taddr0 + (uint32_t)((h >> 1) * 32), r);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) *reinterpret_cast<uint4*>(buf + epi_slot(8 * i + prow, piece)) = Y[h & 1][i];
+    __syncwarp();  // from here on a lane touches only its own row of the buffer, until the stores below
+    if (h + 1 < NH) fetch(h + 1, Y[(h + 1) & 1]);
+    if ((h & 1) == 0) tc_wait_ld();
+    const int col0 = n0 + h * 16;
+#pragma unroll
+    for (int e = 0; e < 16; e += 4) {
+      const uint4 yv = *reinterpret_cast<const uint4*>(buf + epi_slot(lane, e >> 2));
+      const float4 b4 = *reinterpret_cast<const float4*>(g.bias + col0 + e);
+      const int a0 = (h & 1) * 16 + e;
+      float4 o;
+      o.x = fmaf(cs, __uint_as_float(yv.x), co * (__uint_as_float(r[a0 + 0]) + b4.x));
+      o.y = fmaf(cs, __uint_as_float(yv.y), co * (__uint_as_float(r[a0 + 1]) + b4.y));
+      o.z = fmaf(cs, __uint_as_float(yv.z), co * (__uint_as_float(r[a0 + 2]) + b4.z));
+      o.w = fmaf(cs, __uint_as_float(yv.w), co * (__uint_as_float(r[a0 + 3]) + b4.w));
+      *reinterpret_cast<float4*>(buf + epi_slot(lane, e >> 2)) = o;
+    }
+    __syncwarp();
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int row = row_base + 8 * i + prow;
+      const uint4 v = *reinterpret_cast<const uint4*>(buf + epi_slot(8 * i + prow, piece));
+      if (row < m) *reinterpret_cast<uint4*>(g.out_f32 + (size_t)row * g.n_out + col0 + piece * 4) = v;
+    }
+    __syncwarp();
+  }
+}
+
 template <int BN, int EPI>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_w, const GemmArgs g) {
@@ -800,12 +856,13 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
       constexpr int kCols = BN / (kPairEpiWarps / 4);  // this warp's share of the tile's columns
       constexpr int kStagedCols = kCols >= 32 ? kCols : 32;
       const int part = (warp - kEpiWarp0) >> 2;
-      // bf16 outputs of a full tile: global accesses staged through shared memory (warp-uniform choice)
-      const bool staged = EPI != EPI_OUT && kCols % 32 == 0 && n0 + BN <= g.n_out && g.ld_h % 8 == 0;
+      // full tiles: global accesses staged through shared memory (warp-uniform choice)
+      const bool staged = kCols % 32 == 0 && n0 + BN <= g.n_out && (EPI == EPI_OUT ? g.n_out % 4 == 0 : g.ld_h % 8 == 0);
       uint4 R[kStagedCols / 32][4];
       GemmArgs gs = g;  // for the staged path: the bias of this warp's columns comes from shared memory
       if (staged) {
-        epilogue_staged_prefetch<EPI == EPI_OUT ? EPI_IN : EPI, kStagedCols>(g, m0 + quarter * 32, lane, m, n0 + part * kCols, R);
+        if (EPI != EPI_OUT)
+          epilogue_staged_prefetch<EPI == EPI_OUT ? EPI_IN : EPI, kStagedCols>(g, m0 + quarter * 32, lane, m, n0 + part * kCols, R);
         // (fetched while the MMAs run: a bias read behind the accumulator wait costs an L2 round trip per chunk)
         float* sbias = reinterpret_cast<float*>(aux + 256 + kPairEpiWarps * kEpiStageBytes) + (warp - kEpiWarp0) * kCols;
 #pragma unroll
@@ -813,24 +870,27 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
         __syncwarp();
         gs.bias = sbias - (n0 + part * kCols);
       }
-      mbar_wait(accf_bar(acc), acc_phase, dead, g.err);
-      tc_fence_after();
       const int row = m0 + quarter * 32 + lane;
       const bool row_ok = row < m;
       float cs = 0.f, co = 0.f;
       const float* ysrc_row = nullptr;
-      if (EPI == EPI_OUT && row_ok) {
+      if (EPI == EPI_OUT && row_ok) {  // per-row scalars: fetched ahead of the wait as well
         const int step = g.row_step[row];
         cs = g.c_skip[step];
         co = g.c_out[step];
         ysrc_row = g.ysrc + (size_t)(g.row_map ? g.row_map[row] : row) * g.n_out;
       }
+      mbar_wait(accf_bar(acc), acc_phase, dead, g.err);
+      tc_fence_after();
       const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN + part * kCols);
-      if (staged)
-        epilogue_tile_staged<EPI == EPI_OUT ? EPI_IN : EPI, kStagedCols>(
-            gs, taddr, m0 + quarter * 32, lane, m, n0 + part * kCols, aux + 256 + (warp - kEpiWarp0) * kEpiStageBytes, R);
+      uint8_t* buf = aux + 256 + (warp - kEpiWarp0) * kEpiStageBytes;
+      if (staged && EPI == EPI_OUT)
+        epilogue_tile_staged_out<kStagedCols>(gs, taddr, m0 + quarter * 32, lane, m, n0 + part * kCols, buf, cs, co);
+      else if (staged)
+        epilogue_tile_staged<EPI == EPI_OUT ? EPI_IN : EPI, kStagedCols>(gs, taddr, m0 + quarter * 32, lane, m,
+                                                                         n0 + part * kCols, buf, R);
       else
-        epilogue_tile<EPI, kCols, EPI == EPI_OUT>(g, taddr, row, row_ok, n0 + part * kCols, cs, co, ysrc_row);
+        epilogue_tile<EPI, kCols, false>(g, taddr, row, row_ok, n0 + part * kCols, cs, co, ysrc_row);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive_cluster(map_to_cta(acce_bar(acc), 0));
