@@ -505,6 +505,17 @@ def run_ours(args):
         cfgs["cfg1_gmm2d_theta_inf"] = compact_config(torch, AsdSampler, workloads.make("cfg1_gmm2d", window=100), peaks)
         cfgs["cfg2_gauss64_theta_inf"] = compact_config(torch, AsdSampler, workloads.make("cfg2_gauss64", window=1000, chains=64), peaks)
         line["configs"] = cfgs
+        # the batch x window sweep on the cfg-4 denoiser in brief (the full lines: --sweep)
+        if wl.kind == "mlp" and wl.width == 4096 and wl.n_layers == 6 and wl.K == 1000:
+            sweep = {}
+            for b, w in workloads.SWEEP_CELLS:
+                cell = dataclasses.replace(wl, name=f"sweep_b{b}_w{w}", window=w, chains=b)
+                c = compact_config(torch, AsdSampler, cell, peaks, steps=1 if b * w >= 4096 else 2)
+                sweep[cell.name] = {k: c[k] for k in ("samples_per_sec", "rounds_per_sample", "drift_rows_per_sample_over_K",
+                                                      "sequential_gpu_samples_per_sec", "wallclock_speedup_asd")}
+                sweep[cell.name]["dominant_kernel"] = {k: round(v, 4) if isinstance(v, float) else v
+                                                       for k, v in c["dominant_kernel"].items()}
+            line["sweep"] = sweep
     print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()
