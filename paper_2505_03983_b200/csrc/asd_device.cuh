@@ -9,6 +9,15 @@
 
 namespace asd {
 
+// Programmatic dependent launch for the small kernels of a round: the kernel may be scheduled while its predecessor in
+// the stream is still running; it waits for that kernel's completion before it touches anything, and only then lets
+// its own successor be scheduled (a successor that reads a count before its own wait - the weight-streaming GEMM -
+// relies on everything up to the kernel before its predecessor being complete once it runs).
+__device__ __forceinline__ void pdl_wait_then_release() {
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+
 // ---------------------------------------------------------------------------------------------
 // Counter-based randomness (Algorithm 1, "sample u, xi"): Philox4x32-10, counter =
 // (dimension block, step, chain id, tag).

@@ -11,6 +11,23 @@
 
 namespace asd {
 
+// Launch with programmatic stream serialization (see pdl_wait_then_release in asd_device.cuh).
+template <typename... KArgs, typename... Args>
+static void launch_pdl(Ctx* c, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = c->stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+  c->launches++;
+}
+
 // ---------------------------------------------------------------------------------------------
 // Round driver bookkeeping: compact the chains with a < K into the active list and lay out the
 // pass-2 rows (exclusive scan of w - 1).  One block; n is at most a few tens of thousands.
@@ -22,6 +39,7 @@ __global__ void __launch_bounds__(1024) prep_kernel(const int* __restrict__ a, c
                                                     int* __restrict__ step1e, int* __restrict__ idx1,
                                                     int* __restrict__ acc_len, int* __restrict__ first_rej,
                                                     RoundCounters* __restrict__ cnt) {
+  pdl_wait_then_release();
   __shared__ int s_cnt[32], s_rows[32], s_ev[32];
   __shared__ int s_base_cnt, s_base_rows, s_base_ev;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -131,10 +149,9 @@ Lane whole_batch(const Ctx* c) {
 void launch_prep(Ctx* c, const Lane& L, int window) {
   const int* wnd = round_windows(c, window);
   const int la = (c->lookahead && L.act1) ? 1 : 0;
-  prep_kernel<<<1, 1024, 0, c->stream>>>(c->a + L.start, wnd ? wnd + L.start : nullptr, L.n, c->K, window, c->has_v, la,
-                                         L.act, L.row_off, L.step1, L.act1, L.step1e, L.idx1, c->acc_len + L.start,
-                                         c->first_rej + L.start, L.counters);
-  c->launches++;
+  launch_pdl(c, prep_kernel, dim3(1), dim3(1024), 0, c->a + L.start, wnd ? wnd + L.start : nullptr, L.n, c->K, window,
+             c->has_v, la, L.act, L.row_off, L.step1, L.act1, L.step1e, L.idx1, c->acc_len + L.start,
+             c->first_rej + L.start, L.counters);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -201,6 +218,7 @@ __device__ __forceinline__ void draft_store(const DraftArgs& A, int row, int a, 
 }
 
 __global__ void __launch_bounds__(kDraftThreads) draft_kernel(const DraftArgs A) {
+  pdl_wait_then_release();
   __shared__ float4 s_pt[kDraftChunk][kDraftQ];  // noise, then drafted points, per slot of a chunk (parallel form)
   const int p = blockIdx.x;
   if (p >= A.cnt->n_active) return;
@@ -358,8 +376,7 @@ void launch_draft(Ctx* c, const Lane& L, int window, const float* v_base, const 
   A.par = (long long)L.n * ((A.nq + kDraftThreads - 1) / kDraftThreads) < 2ll * c->num_sms;
   const int per_block = A.par ? kDraftQ : kDraftThreads;
   dim3 grid(L.n, (A.nq + per_block - 1) / per_block);  // chains along x (no 65535 limit there)
-  draft_kernel<<<grid, kDraftThreads, 0, c->stream>>>(A);
-  c->launches++;
+  launch_pdl(c, draft_kernel, grid, dim3(kDraftThreads), 0, A);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -474,6 +491,7 @@ __device__ __forceinline__ void slot_partial(const VerifyArgs& A, const float* v
 // needs nothing beyond the first rejection), which is what keeps most of the window's drifts unread.  The skip
 // only saves work: which blocks take it varies from run to run, the result does not.
 __global__ void __launch_bounds__(256, 4) verify_slots_kernel(const VerifyArgs A) {
+  pdl_wait_then_release();
   __shared__ float s_part[kVerifyMaxWarps][2][kVerifyMaxWarps];  // [slot][dot | nrm][warp of team]
   const int p = blockIdx.x;
   if (p >= A.cnt->n_active) return;
@@ -520,6 +538,7 @@ __global__ void __launch_bounds__(256, 4) verify_slots_kernel(const VerifyArgs A
 }
 
 __global__ void __launch_bounds__(256, 3) verify_kernel(const VerifyArgs A) {
+  pdl_wait_then_release();
   __shared__ float s_part[2][kVerifyMaxWarps][2][kVerifyMaxWarps];  // [group parity][slot][dot | nrm][warp of team]
   __shared__ float s_lu[2][kVerifyMaxWarps];                        // [group parity][slot] ln u
   const int p = blockIdx.x;
@@ -747,11 +766,9 @@ void launch_verify(Ctx* c, const Lane& L, int window, bool use_u, const float* G
   A.first_rej = c->first_rej + L.start;
   if (A.horizon > 0) {
     const int S = kVerifyMaxWarps / A.wps;
-    verify_slots_kernel<<<dim3(L.n, (A.horizon + S - 1) / S), 256, 0, c->stream>>>(A);
-    c->launches++;
+    launch_pdl(c, verify_slots_kernel, dim3(L.n, (A.horizon + S - 1) / S), dim3(256), 0, A);
   }
-  verify_kernel<<<L.n, 256, 0, c->stream>>>(A);
-  c->launches++;
+  launch_pdl(c, verify_kernel, dim3(L.n), dim3(256), 0, A);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -759,6 +776,7 @@ void launch_verify(Ctx* c, const Lane& L, int window, bool use_u, const float* G
 // ---------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(128) gmm_kernel(RowSet rs, int d, GmmParams P, const float* __restrict__ tt,
                                                   float* __restrict__ out) {
+  pdl_wait_then_release();
   extern __shared__ float s_logit[];  // [warps][n_comp]
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, wpb = blockDim.x >> 5;
   float* lg = s_logit + warp * P.n_comp;
@@ -772,12 +790,12 @@ void launch_gmm(Ctx* c, const RowSet& rs, float* out) {
   const int threads = 128, wpb = threads / 32;
   int blocks = (rs.n_rows_max + wpb - 1) / wpb;
   blocks = blocks > 8 * c->num_sms ? 8 * c->num_sms : blocks;
-  gmm_kernel<<<blocks, threads, wpb * c->gmm.n_comp * sizeof(float), c->stream>>>(rs, c->d, c->gmm, c->tab.tt, out);
-  c->launches++;
+  launch_pdl(c, gmm_kernel, dim3(blocks), dim3(threads), wpb * c->gmm.n_comp * sizeof(float), rs, c->d, c->gmm, c->tab.tt, out);
 }
 
 __global__ void __launch_bounds__(128) gauss_kernel(RowSet rs, int d, GaussParams P, const float* __restrict__ tt,
                                                     float* __restrict__ out) {
+  pdl_wait_then_release();
   extern __shared__ float s_buf[];  // y[d], w[d]
   float* ys = s_buf;
   float* ws = s_buf + d;
@@ -798,14 +816,14 @@ void launch_gauss(Ctx* c, const RowSet& rs, float* out) {
   if (rs.n_rows_max <= 0) return;
   int blocks = rs.n_rows_max > 16 * c->num_sms ? 16 * c->num_sms : rs.n_rows_max;
   const int threads = c->d >= 128 ? 128 : 64;
-  gauss_kernel<<<blocks, threads, 2 * c->d * sizeof(float), c->stream>>>(rs, c->d, c->gauss, c->tab.tt, out);
-  c->launches++;
+  launch_pdl(c, gauss_kernel, dim3(blocks), dim3(threads), 2 * c->d * sizeof(float), rs, c->d, c->gauss, c->tab.tt, out);
 }
 
 // ---------------------------------------------------------------------------------------------
 // Network input rows for an arbitrary row set: [bf16(c_in y) ; cond ; temb ; 0].
 // ---------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256) pack_kernel(RowSet rs, int d, MlpParams M, const float* __restrict__ c_in) {
+  pdl_wait_then_release();
   const int n_rows = *rs.n_rows_dev;
   for (int r = blockIdx.x; r < n_rows; r += gridDim.x) {
     const float* y = rs.ysrc + (size_t)(rs.row_map ? rs.row_map[r] : r) * d;
@@ -828,8 +846,7 @@ __global__ void __launch_bounds__(256) pack_kernel(RowSet rs, int d, MlpParams M
 void launch_pack(Ctx* c, const RowSet& rs) {
   if (rs.n_rows_max <= 0) return;
   int blocks = rs.n_rows_max > 8 * c->num_sms ? 8 * c->num_sms : rs.n_rows_max;
-  pack_kernel<<<blocks, 256, 0, c->stream>>>(rs, c->d, c->mlp, c->tab.c_in);
-  c->launches++;
+  launch_pdl(c, pack_kernel, dim3(blocks), dim3(256), 0, rs, c->d, c->mlp, c->tab.c_in);
 }
 
 // ---------------------------------------------------------------------------------------------
