@@ -948,3 +948,25 @@ def test_allocation_failure_is_reported_and_leaves_nothing_behind(name, monkeypa
         s.reset(wl.chains, 0, cond=cond)
         y, r, _ = s.sample()
     assert torch.equal(y, y_ref) and torch.equal(r, r_ref)
+
+
+@pytest.mark.parametrize("name,chains", [("cfg1_gmm2d", 20), ("gauss_small", 11)])
+def test_flag_combinations_give_the_same_chains(name, chains):
+    """Closed-form drifts are computed point by point, so neither look-ahead reuse, nor keeping the trajectory, nor the
+    diagnostics, nor which driver runs the loop (chain-resident kernel or per-phase kernels: look-ahead uses the
+    latter) may change a bit of a chain: same samples, rounds, trajectory and prefix histogram for every combination,
+    with fixed and with adaptive windows."""
+    from paper_2505_03983_b200.binding import (FLAG_ADAPTIVE_WINDOW, FLAG_DEBUG_DUMP, FLAG_LOOKAHEAD, FLAG_TRAJECTORY)
+    wl = workloads.make(name, chains=chains)
+    for adaptive in (0, FLAG_ADAPTIVE_WINDOW):
+        ref = None
+        for extra in (0, FLAG_LOOKAHEAD, FLAG_DEBUG_DUMP, FLAG_LOOKAHEAD | FLAG_DEBUG_DUMP):
+            with _sampler(wl, dump=False, flags=FLAG_TRAJECTORY | adaptive | extra) as s:
+                s.reset(chains, 31)
+                y, r, st = s.sample()
+                got = (y, r, s.get_trajectory(), torch.as_tensor(s.prefix_histogram()))
+            if ref is None:
+                ref = got
+            else:
+                for a, b in zip(ref, got):
+                    assert torch.equal(a, b), (adaptive, extra)
