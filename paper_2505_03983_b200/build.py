@@ -9,7 +9,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 LIB = os.path.join(HERE, "libasd_b200.so")
-SOURCES = ["asd_api.cu", "asd_kernels.cu", "asd_resident.cu", "asd_gemm.cu", "asd_static.cu", "asd_schedule.cu"]
+SOURCES = ["asd_api.cu", "asd_kernels.cu", "asd_resident.cu", "asd_gemm.cu", "asd_mlp_fused.cu", "asd_static.cu", "asd_schedule.cu"]
 
 
 def _newest(paths):
@@ -19,6 +19,7 @@ def _newest(paths):
 def build(force: bool = False, verbose: bool = False) -> str:
     srcs = [os.path.join(HERE, "csrc", s) for s in SOURCES]
     deps = srcs + [os.path.join(HERE, "csrc", "asd_internal.h"), os.path.join(HERE, "csrc", "asd_device.cuh"),
+                   os.path.join(HERE, "csrc", "asd_tc.cuh"),
                    os.path.join(ROOT, "include", "asd.h")]
     if not force and os.path.exists(LIB) and os.path.getmtime(LIB) >= _newest(deps):
         return LIB

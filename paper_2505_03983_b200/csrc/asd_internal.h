@@ -245,6 +245,12 @@ void launch_finish(Ctx* c, float* y_out_dev, int* rounds_out_dev);
 // pass: 0 = drift at the current points, 1 = drift at the drafted points, 2 = stand-alone call.
 asd_status mlp_forward(Ctx* c, const RowSet& rs, float* out, int pass);
 void launch_wait_selftest(Ctx* c);  // one bounded wait that must run out (failure-path self-test)
+// 2-D bf16 row-major tensor map [rows, cols], box [box_rows, 64 columns], 128-byte swizzle; cached per context
+bool get_tmap(Ctx* c, const void* ptr, int rows, int cols, int box_rows, CUtensorMap* out);
+void ensure_dynamic_smem(Ctx* c, const void* func, int bytes);  // per-device opt-in to large dynamic shared memory
+// the whole network in one launch (asd_mlp_fused.cu; on request only)
+bool use_fused_mlp(Ctx* c, int m_bound);
+asd_status launch_mlp_fused(Ctx* c, const RowSet& rs, float* out);
 
 // ---- chain-resident round driver for the closed-form drifts (asd_resident.cu) ------------------
 bool resident_supported(const Ctx* c, int window, int* smem_bytes);
