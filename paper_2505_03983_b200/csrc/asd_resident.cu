@@ -61,28 +61,43 @@ __host__ __device__ inline ResidentLayout resident_layout(int kind, int d, int d
   L.tab = o;  o += 5 * wp;                  // eta, sigma, c1, c2, t of the window's steps
   L.extra = o;
   if (kind == ASD_DEN_GAUSS_LINEAR)
-    o += 2 * d * d + 2 * d + wcap * dp;     // Q, Qt, qmu, lam, eigen-coordinates per point (rows of dp)
+    o += 2 * dp * d + 2 * d + wcap * dp;    // Q, Qt (groups of four terms), qmu, lam, eigen-coordinates per point
   else
     o += kResWarps * n_comp + n_comp * (d + 2);  // the warps' logits; means, ln pi, |c|^2
   L.total = o;
   return L;
 }
 
+// The Gaussian's Q and Q^T in shared memory: the four matrix elements that one step of dot_strided4 multiplies sit side by
+// side, element (i, jj) of the matrix at float (i / 4 * d + jj) * 4 + i % 4 (rows past d are zero and never used), so a
+// thread fetches the four terms of its column with one 16-byte load and four neighbouring lanes fetch one term each
+// without a bank conflict.
+struct ResidentGauss {
+  const float4 *Q4, *Qt4;
+  const float *qmu, *lam;
+  float* ws;
+};
+__device__ __forceinline__ ResidentGauss resident_gauss_views(const ResidentArgs& A, const float* sm, const ResidentLayout& L) {
+  ResidentGauss G;
+  G.Q4 = reinterpret_cast<const float4*>(sm + L.extra);
+  G.Qt4 = G.Q4 + (size_t)A.nq * A.d;
+  G.qmu = reinterpret_cast<const float*>(G.Qt4 + (size_t)A.nq * A.d);
+  G.lam = G.qmu + A.d;
+  G.ws = const_cast<float*>(G.lam) + A.d;
+  return G;
+}
+
 // Gaussian posterior mean of n_pts points (rows of dp floats in shared memory) by the whole block.
-// One item = one eigen-coordinate (then one output coordinate) of a group of kPts points: the matrix element is
+// One item = one eigen-coordinate (then one output coordinate) of a group of kPts points: the matrix elements are
 // loaded once for the group and the points' sums run side by side, each in the order of dot_strided4 (four
 // interleaved partial sums), so the bits are those of gauss_coord / gauss_out point by point.
 template <int kPts>
 __device__ __forceinline__ void resident_gauss(const ResidentArgs& A, const float* sm, const ResidentLayout& L,
                                                const float* src, float* dst, int n_pts, const float* s_t) {
   const int tid = threadIdx.x, d = A.d;
-  const float* sQ = sm + L.extra;
-  const float* sQt = sQ + d * d;
-  const float* s_qmu = sQt + d * d;
-  const float* s_lam = s_qmu + d;
-  float* s_ws = const_cast<float*>(s_lam) + d;
+  const ResidentGauss G = resident_gauss_views(A, sm, L);
   const int groups = (n_pts + kPts - 1) / kPts;
-  const int d4 = d & ~3;
+  const int n4 = d >> 2, d4 = d & ~3;
   for (int it = tid; it < groups * d; it += kResThreads) {
     const int pg = it / d, jj = it - pg * d, p0 = pg * kPts;
     const int np = min(kPts, n_pts - p0);
@@ -91,63 +106,103 @@ __device__ __forceinline__ void resident_gauss(const ResidentArgs& A, const floa
 #pragma unroll
     for (int u = 0; u < kPts; ++u) z[u][0] = z[u][1] = z[u][2] = z[u][3] = 0.f;
 #pragma unroll 4
-    for (int i = 0; i < d4; i += 4) {  // four terms per 16-byte (broadcast) load of each point
-      const float q0 = sQ[(size_t)i * d + jj], q1 = sQ[(size_t)(i + 1) * d + jj], q2 = sQ[(size_t)(i + 2) * d + jj],
-                  q3 = sQ[(size_t)(i + 3) * d + jj];
+    for (int i4 = 0; i4 < n4; ++i4) {  // four terms per 16-byte load of the matrix and of each point (broadcast)
+      const float4 q = G.Q4[i4 * d + jj];
 #pragma unroll
       for (int u = 0; u < kPts; ++u) {
-        const float4 yv = *reinterpret_cast<const float4*>(y0 + (size_t)min(u, np - 1) * A.dp + i);
-        z[u][0] = fmaf(q0, yv.x, z[u][0]);
-        z[u][1] = fmaf(q1, yv.y, z[u][1]);
-        z[u][2] = fmaf(q2, yv.z, z[u][2]);
-        z[u][3] = fmaf(q3, yv.w, z[u][3]);
+        const float4 yv = *reinterpret_cast<const float4*>(y0 + (size_t)min(u, np - 1) * A.dp + 4 * i4);
+        z[u][0] = fmaf(q.x, yv.x, z[u][0]);
+        z[u][1] = fmaf(q.y, yv.y, z[u][1]);
+        z[u][2] = fmaf(q.z, yv.z, z[u][2]);
+        z[u][3] = fmaf(q.w, yv.w, z[u][3]);
       }
     }
+    if (d4 < d) {  // the last d mod 4 terms
+      const float4 q = G.Q4[n4 * d + jj];
+      const float qr[3] = {q.x, q.y, q.z};
 #pragma unroll
-    for (int r = 0; r < 3; ++r) {  // the last d mod 4 terms
-      if (d4 + r < d) {
-        const float qv = sQ[(size_t)(d4 + r) * d + jj];
+      for (int r = 0; r < 3; ++r) {
+        if (d4 + r < d) {
 #pragma unroll
-        for (int u = 0; u < kPts; ++u) z[u][r] = fmaf(qv, y0[(size_t)min(u, np - 1) * A.dp + d4 + r], z[u][r]);
+          for (int u = 0; u < kPts; ++u) z[u][r] = fmaf(qr[r], y0[(size_t)min(u, np - 1) * A.dp + d4 + r], z[u][r]);
+        }
       }
     }
-    const float qmu = s_qmu[jj], lam = s_lam[jj];
+    const float qmu = G.qmu[jj], lam = G.lam[jj];
 #pragma unroll
     for (int u = 0; u < kPts; ++u)
-      if (u < np) s_ws[(size_t)(p0 + u) * A.dp + jj] = __fdiv_rn(fmaf(lam, sum4(z[u]), qmu), fmaf(s_t[p0 + u], lam, 1.f));
+      if (u < np) G.ws[(size_t)(p0 + u) * A.dp + jj] = __fdiv_rn(fmaf(lam, sum4(z[u]), qmu), fmaf(s_t[p0 + u], lam, 1.f));
   }
   __syncthreads();
   for (int it = tid; it < groups * d; it += kResThreads) {
     const int pg = it / d, i = it - pg * d, p0 = pg * kPts;
     const int np = min(kPts, n_pts - p0);
-    const float* w0 = s_ws + (size_t)p0 * A.dp;
+    const float* w0 = G.ws + (size_t)p0 * A.dp;
     float m[kPts][4];
 #pragma unroll
     for (int u = 0; u < kPts; ++u) m[u][0] = m[u][1] = m[u][2] = m[u][3] = 0.f;
 #pragma unroll 4
-    for (int jj = 0; jj < d4; jj += 4) {
-      const float q0 = sQt[(size_t)jj * d + i], q1 = sQt[(size_t)(jj + 1) * d + i], q2 = sQt[(size_t)(jj + 2) * d + i],
-                  q3 = sQt[(size_t)(jj + 3) * d + i];
+    for (int j4 = 0; j4 < n4; ++j4) {
+      const float4 q = G.Qt4[j4 * d + i];
 #pragma unroll
       for (int u = 0; u < kPts; ++u) {
-        const float4 wv = *reinterpret_cast<const float4*>(w0 + (size_t)min(u, np - 1) * A.dp + jj);
-        m[u][0] = fmaf(q0, wv.x, m[u][0]);
-        m[u][1] = fmaf(q1, wv.y, m[u][1]);
-        m[u][2] = fmaf(q2, wv.z, m[u][2]);
-        m[u][3] = fmaf(q3, wv.w, m[u][3]);
+        const float4 wv = *reinterpret_cast<const float4*>(w0 + (size_t)min(u, np - 1) * A.dp + 4 * j4);
+        m[u][0] = fmaf(q.x, wv.x, m[u][0]);
+        m[u][1] = fmaf(q.y, wv.y, m[u][1]);
+        m[u][2] = fmaf(q.z, wv.z, m[u][2]);
+        m[u][3] = fmaf(q.w, wv.w, m[u][3]);
       }
     }
+    if (d4 < d) {
+      const float4 q = G.Qt4[n4 * d + i];
+      const float qr[3] = {q.x, q.y, q.z};
 #pragma unroll
-    for (int r = 0; r < 3; ++r) {
-      if (d4 + r < d) {
-        const float qv = sQt[(size_t)(d4 + r) * d + i];
+      for (int r = 0; r < 3; ++r) {
+        if (d4 + r < d) {
 #pragma unroll
-        for (int u = 0; u < kPts; ++u) m[u][r] = fmaf(qv, w0[(size_t)min(u, np - 1) * A.dp + d4 + r], m[u][r]);
+          for (int u = 0; u < kPts; ++u) m[u][r] = fmaf(qr[r], w0[(size_t)min(u, np - 1) * A.dp + d4 + r], m[u][r]);
+        }
       }
     }
 #pragma unroll
     for (int u = 0; u < kPts; ++u)
       if (u < np) dst[(size_t)(p0 + u) * A.dp + i] = sum4(m[u]);
+  }
+  __syncthreads();
+}
+
+// One partial sum of dot_strided4 per lane: lane c of a group of four takes the terms c, c + 4, ... of column `col`
+// in their order, and two exchanges add the partial sums as sum4 does, (s0 + s1) + (s2 + s3) (IEEE addition commutes,
+// so every lane of the group ends with the same bits).  All 32 lanes must call it.
+__device__ __forceinline__ float resident_quarter_dot(const float* M, const float* vec, int d, int col, int c) {
+  const int n4 = d >> 2;
+  float s = 0.f;
+#pragma unroll 8
+  for (int i4 = 0; i4 < n4; ++i4) s = fmaf(M[((size_t)i4 * d + col) * 4 + c], vec[4 * i4 + c], s);
+  if (4 * n4 + c < d) s = fmaf(M[((size_t)n4 * d + col) * 4 + c], vec[4 * n4 + c], s);
+  s = __fadd_rn(s, __shfl_xor_sync(0xffffffffu, s, 1));
+  return __fadd_rn(s, __shfl_xor_sync(0xffffffffu, s, 2));
+}
+
+// The Gaussian posterior mean of ONE point at time t by the whole block: a chain of d / 4 dependent multiply-adds
+// per lane instead of d, with the bits of gauss_coord / gauss_out.
+__device__ __forceinline__ void resident_gauss_one(const ResidentArgs& A, const float* sm, const ResidentLayout& L,
+                                                   const float* src, float* dst, float t) {
+  const int tid = threadIdx.x, d = A.d, c = tid & 3;
+  const ResidentGauss G = resident_gauss_views(A, sm, L);
+  for (int base = 0; base < d; base += kResThreads / 4) {
+    const int jj = base + (tid >> 2), jc = min(jj, d - 1);
+    const float z = resident_quarter_dot(reinterpret_cast<const float*>(G.Q4), src, d, jc, c);
+    if (c == 0 && jj < d) {
+      const float lam = G.lam[jj];
+      G.ws[jj] = __fdiv_rn(fmaf(lam, z, G.qmu[jj]), fmaf(t, lam, 1.f));
+    }
+  }
+  __syncthreads();
+  for (int base = 0; base < d; base += kResThreads / 4) {
+    const int i = base + (tid >> 2), ic = min(i, d - 1);
+    const float m = resident_quarter_dot(reinterpret_cast<const float*>(G.Qt4), G.ws, d, ic, c);
+    if (c == 0 && i < d) dst[i] = m;
   }
   __syncthreads();
 }
@@ -166,6 +221,8 @@ __device__ __forceinline__ void resident_drift(const ResidentArgs& A, const floa
     for (int p = warp; p < n_pts; p += kResWarps)
       gmm_point(src + (size_t)p * A.dp, s_t[p], A.d, P, lg, dst + (size_t)p * A.dp, lane);
     __syncthreads();
+  } else if (n_pts == 1) {
+    resident_gauss_one(A, sm, L, src, dst, s_t[0]);
   } else if (n_pts * A.d <= kResThreads) {
     resident_gauss<1>(A, sm, L, src, dst, n_pts, s_t);  // few points: an item per thread is already all there is
   } else {
@@ -211,13 +268,15 @@ __global__ void __launch_bounds__(kResThreads) resident_kernel(const ResidentArg
   }
   if (KIND == ASD_DEN_GAUSS_LINEAR) {
     float* sQ = sm + L.extra;
-    for (int e = tid; e < d * d; e += kResThreads) {
-      sQ[e] = A.gauss.Q[e];
-      sQ[d * d + e] = A.gauss.Qt[e];
+    const int mat = A.dp * d;
+    for (int e = tid; e < mat; e += kResThreads) {  // element (i, jj) -> (i / 4 * d + jj) * 4 + i % 4
+      const int g = e >> 2, i = 4 * (g / d) + (e & 3), jj = g % d;
+      sQ[e] = i < d ? A.gauss.Q[(size_t)i * d + jj] : 0.f;
+      sQ[mat + e] = i < d ? A.gauss.Qt[(size_t)i * d + jj] : 0.f;
     }
     for (int e = tid; e < d; e += kResThreads) {
-      sQ[2 * d * d + e] = A.gauss.qmu[e];
-      sQ[2 * d * d + d + e] = A.gauss.lam[e];
+      sQ[2 * mat + e] = A.gauss.qmu[e];
+      sQ[2 * mat + d + e] = A.gauss.lam[e];
     }
   } else {
     float* sp = sm + L.extra + kResWarps * A.gmm.n_comp;
@@ -260,9 +319,17 @@ __global__ void __launch_bounds__(kResThreads) resident_kernel(const ResidentArg
     if (tid < nq && w > 1) {
       float4 yh = reinterpret_cast<const float4*>(sy)[tid];
       const float4 v = reinterpret_cast<const float4*>(sv)[tid];
+      float eta_n = s_eta[0], sig_n = s_sig[0];
+      float4 xi_n = sXi4[tid];
       for (int k = 1; k < w; ++k) {
-        const float eta = s_eta[k - 1], sig = s_sig[k - 1];
-        const float4 xi = sXi4[(k - 1) * nq + tid];
+        // the next slot's operands are fetched before this slot's store: the chain then waits on its two multiply-adds only
+        const float eta = eta_n, sig = sig_n;
+        const float4 xi = xi_n;
+        if (k + 1 < w) {
+          eta_n = s_eta[k];
+          sig_n = s_sig[k];
+          xi_n = sXi4[k * nq + tid];
+        }
         yh.x = fmaf(sig, xi.x, fmaf(eta, v.x, yh.x));
         yh.y = fmaf(sig, xi.y, fmaf(eta, v.y, yh.y));
         yh.z = fmaf(sig, xi.z, fmaf(eta, v.z, yh.z));
