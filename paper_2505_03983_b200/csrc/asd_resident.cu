@@ -209,8 +209,9 @@ __device__ __forceinline__ void resident_gauss_one(const ResidentArgs& A, const 
 
 template <int KIND>
 __device__ __forceinline__ void resident_drift(const ResidentArgs& A, const float* sm, const ResidentLayout& L,
-                                               const float* src, float* dst, int n_pts, const float* s_t) {
-  // dst[p] = g(s_t[p], src[p]) for p < n_pts (rows of dp floats; s_t: the points' times); ends with a block barrier
+                                               const float* src, float* dst, int n_pts, const float* s_t, float t_one) {
+  // dst[p] = g(s_t[p], src[p]) for p < n_pts (rows of dp floats; s_t: the points' times); ends with a block barrier.
+  // A single point takes its time from t_one, and s_t is not read before the first block barrier inside.
   if (KIND == ASD_DEN_GMM_ISO) {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     float* lg = const_cast<float*>(sm) + L.extra + warp * A.gmm.n_comp;
@@ -219,10 +220,10 @@ __device__ __forceinline__ void resident_drift(const ResidentArgs& A, const floa
     P.log_pi = P.means + (size_t)A.gmm.n_comp * A.d;
     P.cnorm = P.log_pi + A.gmm.n_comp;
     for (int p = warp; p < n_pts; p += kResWarps)
-      gmm_point(src + (size_t)p * A.dp, s_t[p], A.d, P, lg, dst + (size_t)p * A.dp, lane);
+      gmm_point(src + (size_t)p * A.dp, n_pts == 1 ? t_one : s_t[p], A.d, P, lg, dst + (size_t)p * A.dp, lane);
     __syncthreads();
   } else if (n_pts == 1) {
-    resident_gauss_one(A, sm, L, src, dst, s_t[0]);
+    resident_gauss_one(A, sm, L, src, dst, t_one);
   } else if (n_pts * A.d <= kResThreads) {
     resident_gauss<1>(A, sm, L, src, dst, n_pts, s_t);  // few points: an item per thread is already all there is
   } else {
@@ -290,6 +291,7 @@ __global__ void __launch_bounds__(kResThreads) resident_kernel(const ResidentArg
   int theta_next = A.wnd ? A.wnd[j] : A.window, ema8 = A.wnd ? A.ema8[j] : 0;
   int r_done = 0, n_last = -1, w_first = 0;
   long long rows_total = 0, rows_ver = 0, adv_total = 0;
+  float t_a = A.tab.tt[a];  // t of the current step, carried in a register from round to round
   __syncthreads();
 
   while (a < A.K && r_done < A.max_rounds) {
@@ -312,9 +314,9 @@ __global__ void __launch_bounds__(kResThreads) resident_kernel(const ResidentArg
       const int k = it / nq, q = it - k * nq;
       sXi4[it] = xi4((uint32_t)q, (uint32_t)(a + k + 1), chain, A.keys);
     }
-    __syncthreads();
-    // first model call: v_a = g(t_a, y_a)
-    resident_drift<KIND>(A, sm, L, sy, sv, 1, s_t);
+    // first model call: v_a = g(t_a, y_a).  It reads the state and t_a only, so no barrier separates it from the
+    // noise generation above: its first inner barrier publishes the tables and the noise as well.
+    resident_drift<KIND>(A, sm, L, sy, sv, 1, s_t, t_a);
     // draft: y^_{a+k} = y^_{a+k-1} + eta v_a + sigma xi_{a+k}, k = 1 .. w-1
     if (tid < nq && w > 1) {
       float4 yh = reinterpret_cast<const float4*>(sy)[tid];
@@ -339,7 +341,7 @@ __global__ void __launch_bounds__(kResThreads) resident_kernel(const ResidentArg
     }
     __syncthreads();
     // second model call: the drift at every drafted prefix point
-    if (w > 1) resident_drift<KIND>(A, sm, L, sm + L.yh, sm + L.g, w - 1, s_t + 1);
+    if (w > 1) resident_drift<KIND>(A, sm, L, sm + L.yh, sm + L.g, w - 1, s_t + 1, s_t[1]);
     // Verifier: <xi, delta> and |delta|^2 per slot, one warp per slot, in the reduction order of the verify kernel
     for (int k = 2 + warp; k <= w; k += kResWarps) {
       float dot = 0.f, nrm = 0.f;
@@ -390,6 +392,7 @@ __global__ void __launch_bounds__(kResThreads) resident_kernel(const ResidentArg
     for (int x = 0; x < kResWarps; ++x) first = min(first, s_first[x]);
     const int n = first <= w ? first - 1 : w;  // accepted prefix length
     const int adv = n < w ? n + 1 : w;
+    t_a = s_t[adv];  // = t of step a + adv, the next round's current step
     if (A.dbg_lr) {
       for (int k = 1 + tid; k <= w; k += kResThreads) {
         A.dbg_lu[(size_t)j * A.dbg_stride + k - 1] = s_lu[k];
