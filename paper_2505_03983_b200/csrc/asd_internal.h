@@ -253,7 +253,7 @@ bool use_fused_mlp(Ctx* c, int m_bound);
 asd_status launch_mlp_fused(Ctx* c, const RowSet& rs, float* out);
 
 // ---- chain-resident round driver for the closed-form drifts (asd_resident.cu) ------------------
-bool resident_supported(const Ctx* c, int window, int* smem_bytes);
+bool resident_supported(const Ctx* c, int window, int* smem_bytes, int* k_tab = nullptr);
 // `max_rounds` iterations of Algorithm 1's while loop for every chain (to the end of the grid if large), one launch
 asd_status launch_resident(Ctx* c, int window, bool use_u, int max_rounds);
 

@@ -19,9 +19,11 @@ namespace {
 constexpr int kResThreads = 256;
 constexpr int kResWarps = kResThreads / 32;
 constexpr int kResMaxSmem = 200 * 1024;
+constexpr int kResTabSmem = 100 * 1024;  // with all steps' tables resident: two blocks per SM still fit
 
 struct ResidentArgs {
   int d, dp, nq, vec, K, window, wcap, use_u, all_slots, max_rounds, n;
+  int k_tab;  // K when the tables of all steps stay in shared memory, else 0
   PhiloxKeys keys;
   uint64_t chain_base;
   int* a;
@@ -46,7 +48,9 @@ struct ResidentLayout {
   int y, v, xi, yh, g, lu, dot, nrm, tab, extra, total;
 };
 
-__host__ __device__ inline ResidentLayout resident_layout(int kind, int d, int dp, int wcap, int n_comp) {
+// k_tab > 0: the per-step tables of all k_tab steps stay in shared memory for the whole launch (the window's
+// tables are then views into them); 0: the window's entries are copied in every round.
+__host__ __device__ inline ResidentLayout resident_layout(int kind, int d, int dp, int wcap, int n_comp, int k_tab) {
   ResidentLayout L;
   int o = 0;
   L.y = o;    o += dp;
@@ -58,7 +62,7 @@ __host__ __device__ inline ResidentLayout resident_layout(int kind, int d, int d
   L.lu = o;   o += wp;
   L.dot = o;  o += wp;
   L.nrm = o;  o += wp;
-  L.tab = o;  o += 5 * wp;                  // eta, sigma, c1, c2, t of the window's steps
+  L.tab = o;  o += 5 * (k_tab > 0 ? ((k_tab + 4) & ~3) : wp);  // eta, sigma, c1, c2, t of the window's (or all) steps
   L.extra = o;
   if (kind == ASD_DEN_GAUSS_LINEAR)
     o += 2 * dp * d + 2 * d + wcap * dp;    // Q, Qt (groups of four terms), qmu, lam, eigen-coordinates per point
@@ -244,7 +248,7 @@ __global__ void __launch_bounds__(kResThreads) resident_kernel(const ResidentArg
     if (tid == 0) A.acc_len[j] = -1;
     return;
   }
-  const ResidentLayout L = resident_layout(KIND, A.d, A.dp, A.wcap, A.gmm.n_comp);
+  const ResidentLayout L = resident_layout(KIND, A.d, A.dp, A.wcap, A.gmm.n_comp, A.k_tab);
   float* sy = sm + L.y;
   float* sv = sm + L.v;
   float4* sXi4 = reinterpret_cast<float4*>(sm + L.xi);
@@ -253,12 +257,12 @@ __global__ void __launch_bounds__(kResThreads) resident_kernel(const ResidentArg
   float* s_lu = sm + L.lu;
   float* s_dot = sm + L.dot;
   float* s_nrm = sm + L.nrm;
-  const int wp = (A.wcap + 4) & ~3;
-  float* s_eta = sm + L.tab;   // [k] = eta_{a+k}, k = 0 .. w-1   (step a+k -> a+k+1)
-  float* s_sig = s_eta + wp;   //       sigma_{a+k+1}
-  float* s_c1 = s_sig + wp;
-  float* s_c2 = s_c1 + wp;
-  float* s_t = s_c2 + wp;      // [k] = t_{a+k}, k = 0 .. w
+  const int wp = A.k_tab > 0 ? ((A.k_tab + 4) & ~3) : ((A.wcap + 4) & ~3);
+  float* const tab_eta = sm + L.tab;
+  float* const tab_sig = tab_eta + wp;
+  float* const tab_c1 = tab_sig + wp;
+  float* const tab_c2 = tab_c1 + wp;
+  float* const tab_t = tab_c2 + wp;
   const int nq = A.nq, d = A.d;
   const uint32_t chain = (uint32_t)(A.chain_base + (uint64_t)j);
 
@@ -292,20 +296,36 @@ __global__ void __launch_bounds__(kResThreads) resident_kernel(const ResidentArg
   int r_done = 0, n_last = -1, w_first = 0;
   long long rows_total = 0, rows_ver = 0, adv_total = 0;
   float t_a = A.tab.tt[a];  // t of the current step, carried in a register from round to round
+  if (A.k_tab > 0) {
+    for (int k = tid; k <= A.K; k += kResThreads) {
+      tab_t[k] = A.tab.tt[k];
+      if (k < A.K) {
+        tab_eta[k] = A.tab.eta[k];
+        tab_sig[k] = A.tab.sig[k];
+        tab_c1[k] = A.tab.c1[k];
+        tab_c2[k] = A.tab.c2[k];
+      }
+    }
+  }
   __syncthreads();
 
   while (a < A.K && r_done < A.max_rounds) {
     const int theta = A.wnd ? max(1, min(theta_next, A.window)) : A.window;
     const int w = min(theta, A.K - a);  // Algorithm 1: b = min(K, a + theta)
     if (r_done == 0) w_first = w;
-    // the window's per-step tables: one trip to global memory per round, under the noise generation
-    for (int k = tid; k <= w; k += kResThreads) {
-      s_t[k] = A.tab.tt[a + k];
-      if (k < w) {
-        s_eta[k] = A.tab.eta[a + k];
-        s_sig[k] = A.tab.sig[a + k];
-        s_c1[k] = A.tab.c1[a + k];
-        s_c2[k] = A.tab.c2[a + k];
+    // the window's per-step tables: [k] = eta_{a+k}, sigma_{a+k+1}, c1, c2 for k = 0 .. w-1 and t_{a+k} for k = 0 .. w;
+    // views into the resident tables, or one trip to global memory per round under the noise generation
+    const int off = A.k_tab > 0 ? a : 0;
+    const float *s_eta = tab_eta + off, *s_sig = tab_sig + off, *s_c1 = tab_c1 + off, *s_c2 = tab_c2 + off, *s_t = tab_t + off;
+    if (A.k_tab == 0) {
+      for (int k = tid; k <= w; k += kResThreads) {
+        tab_t[k] = A.tab.tt[a + k];
+        if (k < w) {
+          tab_eta[k] = A.tab.eta[a + k];
+          tab_sig[k] = A.tab.sig[a + k];
+          tab_c1[k] = A.tab.c1[a + k];
+          tab_c2[k] = A.tab.c2[a + k];
+        }
       }
     }
     // ln u and xi of every slot of the window (counter-based: the same values in every round that reaches a step)
@@ -491,22 +511,32 @@ __global__ void resident_begin_kernel(RoundCounters* cnt) {
 
 // Whether the chain-resident kernel can serve this context (closed-form drift, one-warp reduction teams,
 // the window's working set fits shared memory); *smem_bytes receives the dynamic shared memory it needs.
-bool resident_supported(const Ctx* c, int window, int* smem_bytes) {
+bool resident_supported(const Ctx* c, int window, int* smem_bytes, int* k_tab) {
   if (c->kind != ASD_DEN_GMM_ISO && c->kind != ASD_DEN_GAUSS_LINEAR) return false;
   if (c->lookahead) return false;
   const int nq = (c->d + 3) / 4;
   if (nq >= 512 || nq > kResThreads) return false;
-  const ResidentLayout L = resident_layout(c->kind, c->d, 4 * nq, std::max(window, 1), c->gmm.n_comp);
-  const long long bytes = (long long)L.total * 4;
+  ResidentLayout L = resident_layout(c->kind, c->d, 4 * nq, std::max(window, 1), c->gmm.n_comp, 0);
+  long long bytes = (long long)L.total * 4;
   if (bytes > kResMaxSmem) return false;
+  if (k_tab) {
+    // all K steps' tables resident when the block still leaves room for a second one on the SM
+    *k_tab = 0;
+    L = resident_layout(c->kind, c->d, 4 * nq, std::max(window, 1), c->gmm.n_comp, c->K);
+    if ((long long)L.total * 4 <= kResTabSmem) {
+      *k_tab = c->K;
+      bytes = (long long)L.total * 4;
+    }
+  }
   if (smem_bytes) *smem_bytes = (int)bytes;
   return true;
 }
 
 // `max_rounds` iterations of Algorithm 1's while loop (or to the end of the grid) for every chain, one launch.
 asd_status launch_resident(Ctx* c, int window, bool use_u, int max_rounds) {
-  int smem = 0;
-  if (!resident_supported(c, window, &smem)) return ASD_ERR_UNSUPPORTED;
+  int smem = 0, k_tab = 0;
+  // a launch of a single round (lock-step use) keeps the per-round copy of the window's tables
+  if (!resident_supported(c, window, &smem, max_rounds > 1 ? &k_tab : nullptr)) return ASD_ERR_UNSUPPORTED;
   if (c->n <= 0) return ASD_OK;
   ResidentArgs A{};
   A.d = c->d;
@@ -514,6 +544,7 @@ asd_status launch_resident(Ctx* c, int window, bool use_u, int max_rounds) {
   A.dp = 4 * A.nq;
   A.vec = (c->d % 4 == 0);
   A.K = c->K;
+  A.k_tab = k_tab;
   A.window = window;
   A.wcap = std::max(window, 1);
   A.use_u = use_u ? 1 : 0;
