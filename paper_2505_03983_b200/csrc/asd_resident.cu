@@ -65,7 +65,7 @@ __host__ __device__ inline ResidentLayout resident_layout(int kind, int d, int d
   L.tab = o;  o += 5 * (k_tab > 0 ? ((k_tab + 4) & ~3) : wp);  // eta, sigma, c1, c2, t of the window's (or all) steps
   L.extra = o;
   if (kind == ASD_DEN_GAUSS_LINEAR)
-    o += 2 * dp * d + 2 * d + wcap * dp;    // Q, Qt (groups of four terms), qmu, lam, eigen-coordinates per point
+    o += 2 * dp * d + ((2 * d + 3) & ~3) + wcap * dp;  // Q, Qt (groups of four terms), qmu, lam (padded to 16 bytes), eigen-coordinates per point
   else
     o += kResWarps * n_comp + n_comp * (d + 2);  // the warps' logits; means, ln pi, |c|^2
   L.total = o;
@@ -87,7 +87,7 @@ __device__ __forceinline__ ResidentGauss resident_gauss_views(const ResidentArgs
   G.Qt4 = G.Q4 + (size_t)A.nq * A.d;
   G.qmu = reinterpret_cast<const float*>(G.Qt4 + (size_t)A.nq * A.d);
   G.lam = G.qmu + A.d;
-  G.ws = const_cast<float*>(G.lam) + A.d;
+  G.ws = const_cast<float*>(G.qmu) + ((2 * A.d + 3) & ~3);  // rows of dp floats, read 16 bytes at a time
   return G;
 }
 

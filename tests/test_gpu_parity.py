@@ -818,7 +818,7 @@ def test_context_created_on_a_busy_side_stream():
 # ------------------------------------------------------------------ chain-resident kernel (closed-form drifts)
 @pytest.mark.parametrize("name,chains,kw", [("cfg1_gmm2d", 16, {}), ("cfg2_gauss64", 40, {"K": 300}), ("gmm_odd", 9, {}),
                                             ("gauss_small", 11, {}), ("cfg1_gmm2d", 7, {"K": 200, "window": 200}),
-                                            ("gauss_small", 3, {"window": 1})])
+                                            ("gauss_small", 3, {"window": 1}), ("gauss_odd", 5, {})])
 @pytest.mark.parametrize("flags", ["plain", "adaptive", "all_slots"])
 def test_resident_kernel_equals_per_phase_kernels(name, chains, kw, flags, monkeypatch):
     """asd_sample / asd_sequential_ddpm on the closed-form drifts run Algorithm 1's while loop inside one launch
@@ -856,7 +856,8 @@ def test_resident_kernel_equals_per_phase_kernels(name, chains, kw, flags, monke
 
 
 @pytest.mark.parametrize("name,chains,rounds,kw", [("cfg1_gmm2d", 16, 60, {}), ("gmm_odd", 9, 30, {}), ("gauss_small", 11, 40, {}),
-                                                   ("cfg2_gauss64", 24, 12, {}), ("cfg1_gmm2d", 5, 12, {"K": 300, "window": 300})])
+                                                   ("cfg2_gauss64", 24, 12, {}), ("cfg1_gmm2d", 5, 12, {"K": 300, "window": 300}),
+                                                   ("gauss_odd", 5, 20, {})])
 @pytest.mark.parametrize("adaptive", [False, True])
 def test_lockstep_resident_kernel_rounds(name, chains, rounds, kw, adaptive, monkeypatch):
     """The chain-resident kernel limited to one round per launch (ASD_RESIDENT=2 routes asd_round through it),

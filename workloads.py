@@ -193,6 +193,9 @@ def make(name: str, *, chains: Optional[int] = None, K: Optional[int] = None,
         return _gmm(name, 5, 3, 0.5, ov(K, 50), ov(window, 7), ov(chains, 9), s)
     if name == "gauss_small":
         return _gauss(name, 12, ov(K, 80), ov(window, 5), ov(chains, 11), s)
+    if name == "gauss_odd":
+        # an odd dimension: a ragged last float4 group and parameter vectors of odd length
+        return _gauss(name, 37, ov(K, 60), ov(window, 6), ov(chains, 5), s)
     raise KeyError(name)
 
 
