@@ -328,8 +328,7 @@ __global__ void __launch_bounds__(kResThreads) resident_kernel(const ResidentArg
         }
       }
     }
-    // ln u and xi of every slot of the window (counter-based: the same values in every round that reaches a step)
-    for (int k = 1 + tid; k <= w; k += kResThreads) s_lu[k] = A.use_u ? ln_u((uint32_t)(a + k), chain, A.keys) : 0.f;
+    // xi of every slot of the window (counter-based: the same values in every round that reaches a step)
     for (int it = tid; it < w * nq; it += kResThreads) {
       const int k = it / nq, q = it - k * nq;
       sXi4[it] = xi4((uint32_t)q, (uint32_t)(a + k + 1), chain, A.keys);
@@ -337,6 +336,9 @@ __global__ void __launch_bounds__(kResThreads) resident_kernel(const ResidentArg
     // first model call: v_a = g(t_a, y_a).  It reads the state and t_a only, so no barrier separates it from the
     // noise generation above: its first inner barrier publishes the tables and the noise as well.
     resident_drift<KIND>(A, sm, L, sy, sv, 1, s_t, t_a);
+    // ln u of every slot, by the block's last threads while its first ones draft (the accept tests read it two
+    // barriers later; in the noise phase it would make one warp the straggler of the first barrier)
+    for (int k = 1 + (kResThreads - 1 - tid); k <= w; k += kResThreads) s_lu[k] = A.use_u ? ln_u((uint32_t)(a + k), chain, A.keys) : 0.f;
     // draft: y^_{a+k} = y^_{a+k-1} + eta v_a + sigma xi_{a+k}, k = 1 .. w-1
     if (tid < nq && w > 1) {
       float4 yh = reinterpret_cast<const float4*>(sy)[tid];
@@ -449,7 +451,7 @@ __global__ void __launch_bounds__(kResThreads) resident_kernel(const ResidentArg
         if (b0 + 3 >= d) o.w = 0.f;
       }
     }
-    __syncthreads();  // every reader of the old state is done
+    // (since the draft, the old state has been read by its own thread only: no barrier before the write)
     if (tid < nq) reinterpret_cast<float4*>(sy)[tid] = o;
     __syncthreads();
     if (A.traj) {
