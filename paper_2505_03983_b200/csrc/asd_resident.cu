@@ -91,6 +91,17 @@ __device__ __forceinline__ ResidentGauss resident_gauss_views(const ResidentArgs
   return G;
 }
 
+// Two IEEE fused multiply-adds in one instruction (sm_100 packed fp32): acc.x = fma(a.x, b.x, acc.x), acc.y likewise;
+// each half rounds exactly as fmaf does.
+__device__ __forceinline__ void fma2(float& acc_x, float& acc_y, float ax, float ay, float bx, float by) {
+  asm("{\n\t.reg .b64 pa, pb, pc;\n\t"
+      "mov.b64 pa, {%2, %3};\n\tmov.b64 pb, {%4, %5};\n\tmov.b64 pc, {%0, %1};\n\t"
+      "fma.rn.f32x2 pc, pa, pb, pc;\n\t"
+      "mov.b64 {%0, %1}, pc;\n\t}"
+      : "+f"(acc_x), "+f"(acc_y)
+      : "f"(ax), "f"(ay), "f"(bx), "f"(by));
+}
+
 // Gaussian posterior mean of n_pts points (rows of dp floats in shared memory) by the whole block.
 // One item = one eigen-coordinate (then one output coordinate) of a group of kPts points: the matrix elements are
 // loaded once for the group and the points' sums run side by side, each in the order of dot_strided4 (four
@@ -115,10 +126,8 @@ __device__ __forceinline__ void resident_gauss(const ResidentArgs& A, const floa
 #pragma unroll
       for (int u = 0; u < kPts; ++u) {
         const float4 yv = *reinterpret_cast<const float4*>(y0 + (size_t)min(u, np - 1) * A.dp + 4 * i4);
-        z[u][0] = fmaf(q.x, yv.x, z[u][0]);
-        z[u][1] = fmaf(q.y, yv.y, z[u][1]);
-        z[u][2] = fmaf(q.z, yv.z, z[u][2]);
-        z[u][3] = fmaf(q.w, yv.w, z[u][3]);
+        fma2(z[u][0], z[u][1], q.x, q.y, yv.x, yv.y);
+        fma2(z[u][2], z[u][3], q.z, q.w, yv.z, yv.w);
       }
     }
     if (d4 < d) {  // the last d mod 4 terms
@@ -151,10 +160,8 @@ __device__ __forceinline__ void resident_gauss(const ResidentArgs& A, const floa
 #pragma unroll
       for (int u = 0; u < kPts; ++u) {
         const float4 wv = *reinterpret_cast<const float4*>(w0 + (size_t)min(u, np - 1) * A.dp + 4 * j4);
-        m[u][0] = fmaf(q.x, wv.x, m[u][0]);
-        m[u][1] = fmaf(q.y, wv.y, m[u][1]);
-        m[u][2] = fmaf(q.z, wv.z, m[u][2]);
-        m[u][3] = fmaf(q.w, wv.w, m[u][3]);
+        fma2(m[u][0], m[u][1], q.x, q.y, wv.x, wv.y);
+        fma2(m[u][2], m[u][3], q.z, q.w, wv.z, wv.w);
       }
     }
     if (d4 < d) {
