@@ -614,11 +614,11 @@ gemm_skinny_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
           const int lr = lr0 + u * kRowStep;
           if (lr < m) {
             const int row = row0 + lr;
-            float x = acc[u] + bias;
             if (EPI == EPI_OUT) {
+              const float x = acc[u] + bias;
               g.out_f32[(size_t)row * g.n_out + n] = fmaf(cs[u], opnd[u], co[u] * x);
             } else {
-              if (EPI == EPI_HID) x = opnd[u] + silu(x);
+              const float x = EPI == EPI_HID ? hid_tail(acc[u], bias, opnd[u]) : __fadd_rn(acc[u], bias);
               g.out_bf16[(size_t)row * g.ld_h + n] = __float2bfloat16_rn(x);
             }
           }

@@ -220,9 +220,59 @@ struct Cfg {
   static constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
 };
 
-// SiLU on the un-rounded fp32 accumulator; ex2.approx and rcp.approx (relative error ~2^-22, far below
-// the bf16 rounding that follows).
-__device__ __forceinline__ float silu(float z) { return __fdividef(z, 1.0f + __expf(-z)); }
+// The tail of a residual layer on the un-rounded fp32 accumulator: z = acc + bias, then resid + z sigmoid(z) with
+// sigmoid(z) = 1 / (1 + 2^(-z log2 e)) from ex2.approx and rcp.approx (relative error ~2^-22, far below the bf16
+// rounding that follows; z -> -inf gives 2^(+inf) = inf, 1 / inf = 0, the right limit).  Every step is spelled out
+// (no contraction left to the compiler), so the scalar form and the packed form below, which does two columns per
+// instruction with sm_100's two-way fp32 add / mul / fma, return the same bits in every kernel that uses them.
+constexpr float kNegLog2e = -1.4426950408889634f;
+__device__ __forceinline__ float ex2_approx(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ float rcp_approx(float x) {
+  float y;
+  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ float hid_tail(float acc, float bias, float resid) {
+  const float z = __fadd_rn(acc, bias);
+  const float e = ex2_approx(__fmul_rn(z, kNegLog2e));
+  const float r = rcp_approx(__fadd_rn(1.0f, e));
+  return __fmaf_rn(z, r, resid);
+}
+__device__ __forceinline__ float2 add2(float2 a, float2 b) {
+  float2 c;
+  asm("{\n\t.reg .b64 pa, pb, pc;\n\tmov.b64 pa, {%2, %3};\n\tmov.b64 pb, {%4, %5};\n\t"
+      "add.rn.f32x2 pc, pa, pb;\n\tmov.b64 {%0, %1}, pc;\n\t}"
+      : "=f"(c.x), "=f"(c.y)
+      : "f"(a.x), "f"(a.y), "f"(b.x), "f"(b.y));
+  return c;
+}
+__device__ __forceinline__ float2 mul2(float2 a, float2 b) {
+  float2 c;
+  asm("{\n\t.reg .b64 pa, pb, pc;\n\tmov.b64 pa, {%2, %3};\n\tmov.b64 pb, {%4, %5};\n\t"
+      "mul.rn.f32x2 pc, pa, pb;\n\tmov.b64 {%0, %1}, pc;\n\t}"
+      : "=f"(c.x), "=f"(c.y)
+      : "f"(a.x), "f"(a.y), "f"(b.x), "f"(b.y));
+  return c;
+}
+__device__ __forceinline__ float2 fma2(float2 a, float2 b, float2 c) {
+  float2 d;
+  asm("{\n\t.reg .b64 pa, pb, pc, pd;\n\tmov.b64 pa, {%2, %3};\n\tmov.b64 pb, {%4, %5};\n\tmov.b64 pc, {%6, %7};\n\t"
+      "fma.rn.f32x2 pd, pa, pb, pc;\n\tmov.b64 {%0, %1}, pd;\n\t}"
+      : "=f"(d.x), "=f"(d.y)
+      : "f"(a.x), "f"(a.y), "f"(b.x), "f"(b.y), "f"(c.x), "f"(c.y));
+  return d;
+}
+// hid_tail on two neighbouring columns
+__device__ __forceinline__ float2 hid_tail2(float2 acc, float2 bias, float2 resid) {
+  const float2 z = add2(acc, bias);
+  const float2 t = mul2(z, make_float2(kNegLog2e, kNegLog2e));
+  const float2 den = add2(make_float2(1.0f, 1.0f), make_float2(ex2_approx(t.x), ex2_approx(t.y)));
+  return fma2(z, make_float2(rcp_approx(den.x), rcp_approx(den.y)), resid);
+}
 
 // Epilogue of 32 consecutive accumulator columns [col0, col0 + 32) of one output row held by this
 // thread: bias, then the layer's fused tail, then the store (16-byte vectors where the shape allows).
@@ -263,17 +313,18 @@ __device__ __forceinline__ void epilogue_chunk(const GemmArgs& g, int row, int c
         const float4 b0 = *reinterpret_cast<const float4*>(g.bias + col0 + e);
         const float4 b1 = *reinterpret_cast<const float4*>(g.bias + col0 + e + 4);
         const float bb[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
-#pragma unroll
-        for (int u = 0; u < 8; ++u) x[u] = __uint_as_float(r[e + u]) + bb[u];
         if (EPI == EPI_HID) {
           const uint4 rv = *reinterpret_cast<const uint4*>(rrow + col0 + e);
           const __nv_bfloat162* rp = reinterpret_cast<const __nv_bfloat162*>(&rv);
 #pragma unroll
           for (int u = 0; u < 4; ++u) {
             const float2 rf = __bfloat1622float2(rp[u]);
-            x[2 * u] = rf.x + silu(x[2 * u]);
-            x[2 * u + 1] = rf.y + silu(x[2 * u + 1]);
+            x[2 * u] = hid_tail(__uint_as_float(r[e + 2 * u]), bb[2 * u], rf.x);
+            x[2 * u + 1] = hid_tail(__uint_as_float(r[e + 2 * u + 1]), bb[2 * u + 1], rf.y);
           }
+        } else {
+#pragma unroll
+          for (int u = 0; u < 8; ++u) x[u] = __fadd_rn(__uint_as_float(r[e + u]), bb[u]);
         }
         uint4 ov;
         __nv_bfloat162* op = reinterpret_cast<__nv_bfloat162*>(&ov);
@@ -286,8 +337,8 @@ __device__ __forceinline__ void epilogue_chunk(const GemmArgs& g, int row, int c
       for (int e = 0; e < 32; ++e) {
         const int col = col0 + e;
         if (col < g.n_out) {
-          float x = __uint_as_float(r[e]) + g.bias[col];
-          if (EPI == EPI_HID) x = __bfloat162float(rrow[col]) + silu(x);
+          const float x = EPI == EPI_HID ? hid_tail(__uint_as_float(r[e]), g.bias[col], __bfloat162float(rrow[col]))
+                                         : __fadd_rn(__uint_as_float(r[e]), g.bias[col]);
           orow[col] = __float2bfloat16_rn(x);
         }
       }
@@ -341,17 +392,18 @@ __device__ __forceinline__ void epi_apply(const GemmArgs& g, int row, int col0, 
       const float4 b0 = *reinterpret_cast<const float4*>(g.bias + col0 + e);
       const float4 b1 = *reinterpret_cast<const float4*>(g.bias + col0 + e + 4);
       const float bb[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
-#pragma unroll
-      for (int u = 0; u < 8; ++u) x[u] = __uint_as_float(r[e + u]) + bb[u];
       if (EPI == EPI_HID) {
         const uint4 rv = op.v[e >> 3];
         const __nv_bfloat162* rp = reinterpret_cast<const __nv_bfloat162*>(&rv);
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
           const float2 rf = __bfloat1622float2(rp[u]);
-          x[2 * u] = rf.x + silu(x[2 * u]);
-          x[2 * u + 1] = rf.y + silu(x[2 * u + 1]);
+          x[2 * u] = hid_tail(__uint_as_float(r[e + 2 * u]), bb[2 * u], rf.x);
+          x[2 * u + 1] = hid_tail(__uint_as_float(r[e + 2 * u + 1]), bb[2 * u + 1], rf.y);
         }
+      } else {
+#pragma unroll
+        for (int u = 0; u < 8; ++u) x[u] = __fadd_rn(__uint_as_float(r[e + u]), bb[u]);
       }
       uint4 ov;
       __nv_bfloat162* op2 = reinterpret_cast<__nv_bfloat162*>(&ov);
@@ -445,16 +497,23 @@ __device__ __forceinline__ void epi_staged_chunk(const GemmArgs& g, uint32_t tad
       const float4 b0 = *reinterpret_cast<const float4*>(g.bias + col0 + e);
       const float4 b1 = *reinterpret_cast<const float4*>(g.bias + col0 + e + 4);
       const float bb[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
-#pragma unroll
-      for (int u = 0; u < 8; ++u) x[u] = __uint_as_float(r[e + u]) + bb[u];
       if (EPI == EPI_HID) {
         const uint4 rv = *reinterpret_cast<const uint4*>(buf + epi_slot(lane, e >> 3));
         const __nv_bfloat162* rp = reinterpret_cast<const __nv_bfloat162*>(&rv);
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
-          const float2 rf = __bfloat1622float2(rp[u]);
-          x[2 * u] = rf.x + silu(x[2 * u]);
-          x[2 * u + 1] = rf.y + silu(x[2 * u + 1]);
+          const float2 o2 = hid_tail2(make_float2(__uint_as_float(r[e + 2 * u]), __uint_as_float(r[e + 2 * u + 1])),
+                                      make_float2(bb[2 * u], bb[2 * u + 1]), __bfloat1622float2(rp[u]));
+          x[2 * u] = o2.x;
+          x[2 * u + 1] = o2.y;
+        }
+      } else {
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const float2 o2 = add2(make_float2(__uint_as_float(r[e + 2 * u]), __uint_as_float(r[e + 2 * u + 1])),
+                                 make_float2(bb[2 * u], bb[2 * u + 1]));
+          x[2 * u] = o2.x;
+          x[2 * u + 1] = o2.y;
         }
       }
       uint4 ov;
