@@ -33,7 +33,7 @@ DEFAULT_WORKLOAD = "sweep_b512_w64"   # cfg-4 denoiser, 512 chains x window 64, 
 # dram__bytes_read.sum + dram__bytes_write.sum of one pass-2 hidden-layer launch of gemm_pair_kernel<256, EPI_HID>
 # at full row count, from one ncu capture of that kernel; set an entry to None when the kernel changes, until the
 # counters are taken again
-NCU_TRAFFIC_BYTES_PER_LAUNCH = {"sweep_b512_w64": 390_400_000 + 246_830_000}
+NCU_TRAFFIC_BYTES_PER_LAUNCH = {"sweep_b512_w64": 408_912_896 + 248_380_928}
 METRIC = "samples_per_sec"
 UNIT = "samples/s"
 
